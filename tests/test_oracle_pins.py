@@ -1,0 +1,371 @@
+"""Pins for the CPU oracle: brute force, closed forms, invariants, special cases.
+
+None of these tests touches the CUDA library.  Each pin names the passage of
+the paper (arXiv 2106.09236) that fixes the expected value.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import brute
+from oracle import psattn_oracle as orc
+from paper_2106_09236_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rand(B, H, T, d, seed, n_cols, lengths=None):
+    rng = np.random.default_rng(seed)
+    Q = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    K = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    V = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    if lengths is None:
+        lengths = np.full(B, T, dtype=np.int32)
+    idx = np.zeros((B, T, n_cols), dtype=np.int32)
+    for b in range(B):
+        L = int(lengths[b])
+        idx[b, :L] = rng.integers(0, L, size=(L, n_cols))
+    return Q, K, V, idx, np.asarray(lengths, dtype=np.int32)
+
+
+# ---- sample-size rule (Sec. 3.2: L~ = r_sample ln L) -----------------------------------
+
+def test_count_golden_table():
+    """The workload definitions state the counts 25/32/35/46 for c = 5."""
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "sample_counts.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) >= 4
+    for T, c, n in rows:
+        assert orc.count(float(c), int(T)) == int(n)
+
+
+def test_count_closed_form_and_clamps():
+    for L in range(1, 700):
+        for c in (0.3, 1.0, 5.0, 40.0):
+            want = min(L, max(1, math.ceil(c * math.log(L))))
+            assert orc.count(c, L) == want
+    assert orc.count(5.0, 1) == 1          # ln 1 = 0 -> clamp up to one sample
+    assert orc.count(5.0, 3) == 3          # ceil(5.49) = 6 -> clamp down to len
+    assert orc.count(5.0, 0) == 0
+
+
+# ---- P1: whole oracle vs brute force ----------------------------------------------------
+
+@pytest.mark.parametrize("T", [1, 2, 3, 5, 8, 17, 32])
+@pytest.mark.parametrize("fill", ["mean_v", "own_v"])
+def test_brute_force_tiny(T, fill):
+    B, H, d, c = 2, 2, 8, 1.5
+    lengths = np.array([T, max(1, T - 2)], dtype=np.int32)
+    ncol = max(brute.n_count(c, T), 1)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 100 + T, ncol, lengths)
+    O, sel, M = orc.forward(Q, K, V, idx, lengths, c=c, fill=fill)
+    Ob, selb, Mb = brute.forward(Q, K, V, idx, lengths, c, fill=fill)
+    np.testing.assert_allclose(M, Mb, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(O, Ob, rtol=0, atol=1e-12)
+    k = 0
+    for b in range(B):
+        for h in range(H):
+            got = [int(x) for x in sel[b, h] if x >= 0]
+            assert got == selb[k], (b, h)
+            assert got == sorted(got)
+            k += 1
+
+
+def test_brute_force_d64_with_duplicates():
+    """d = 64 as in the model; sample rows with forced duplicates (multiplicity in the mean)."""
+    B, H, T, d, c = 1, 2, 24, 64, 2.0
+    ncol = brute.n_count(c, T)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 7, ncol)
+    idx[:, :, 1] = idx[:, :, 0]            # every row has a duplicate
+    idx[:, 3, :] = 5                       # one row is a single key repeated
+    O, sel, M = orc.forward(Q, K, V, idx, lengths, c=c)
+    Ob, selb, Mb = brute.forward(Q, K, V, idx, lengths, c)
+    np.testing.assert_allclose(M, Mb, atol=1e-12)
+    np.testing.assert_allclose(O, Ob, atol=1e-12)
+    assert M[0, 0, 3] == 0.0 and M[0, 1, 3] == 0.0
+
+
+# ---- P2: u = len  ==> dense softmax attention (Eq. 6) ------------------------------------
+
+def test_all_selected_equals_dense_attention():
+    import torch
+    B, H, T, d = 2, 3, 40, 16
+    lengths = np.array([40, 29], dtype=np.int32)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 11, 6, lengths)
+    O, sel, _ = orc.forward(Q, K, V, idx, lengths, c=1.0, u_override=T)
+    Od = orc.dense(Q, K, V, lengths)
+    np.testing.assert_allclose(O, Od, atol=1e-13)
+    for b in range(B):
+        L = int(lengths[b])
+        assert [int(x) for x in sel[b, 0] if x >= 0] == list(range(L))
+        q = torch.from_numpy(Q[b, :, :L]).double()
+        k = torch.from_numpy(K[b, :, :L]).double()
+        v = torch.from_numpy(V[b, :, :L]).double()
+        ref = torch.nn.functional.scaled_dot_product_attention(q, k, v).numpy()
+        np.testing.assert_allclose(O[b, :, :L], ref, atol=1e-10)
+        assert np.all(O[b, :, L:] == 0.0)
+
+
+# ---- P3: non-selected rows are the column mean of V -------------------------------------
+
+def test_non_selected_rows_equal_mean_v():
+    B, H, T, d, c = 2, 2, 50, 8, 1.0
+    lengths = np.array([50, 33], dtype=np.int32)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 12, brute.n_count(c, T), lengths)
+    O, sel, _ = orc.forward(Q, K, V, idx, lengths, c=c)
+    vb = orc.mean_v(V, lengths)
+    for b in range(B):
+        L = int(lengths[b])
+        for h in range(H):
+            np.testing.assert_allclose(vb[b, h], V[b, h, :L].astype(np.float64).mean(axis=0),
+                                       atol=1e-14)
+            chosen = set(int(x) for x in sel[b, h] if x >= 0)
+            assert len(chosen) == brute.n_count(c, L)
+            for i in range(L):
+                if i not in chosen:
+                    np.testing.assert_array_equal(O[b, h, i], vb[b, h])
+
+
+def test_own_value_fill_is_eq12_as_printed():
+    B, H, T, d, c = 1, 2, 30, 8, 1.0
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 13, brute.n_count(c, T))
+    O, sel, _ = orc.forward(Q, K, V, idx, lengths, c=c, fill="own_v")
+    for h in range(H):
+        chosen = set(int(x) for x in sel[0, h] if x >= 0)
+        for i in range(T):
+            if i not in chosen:
+                np.testing.assert_array_equal(O[0, h, i], V[0, h, i].astype(np.float64))
+
+
+# ---- P4: M >= 0, and M == 0 for a constant-score query ---------------------------------
+
+def test_measure_nonnegative_and_zero_for_constant_scores():
+    B, H, T, d = 1, 2, 64, 64
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 14, 21)
+    Q[0, 0, 7] = 0.0                        # q = 0 -> every score 0
+    idx[0, 9, :] = 4                        # one key repeated -> constant scores
+    M = orc.measure(Q, K, idx, lengths, U_override=21)
+    assert np.all(M >= 0.0)
+    assert M[0, 0, 7] == 0.0
+    assert M[0, 0, 9] == 0.0 and M[0, 1, 9] == 0.0
+    K2 = np.broadcast_to(K[:, :, :1], K.shape).copy()   # all key rows equal
+    M2 = orc.measure(Q, K2, idx, lengths, U_override=21)
+    assert np.all(M2 == 0.0)
+
+
+# ---- P5: closed form with orthogonal keys -------------------------------------------------
+
+def test_measure_closed_form_orthogonal_keys():
+    """K rows orthogonal with norm rho, q = alpha k_p, p drawn m times out of U:
+    scores are alpha rho^2/sqrt(d) on p and 0 elsewhere, so
+    M = (alpha rho^2 / sqrt(d)) (1 - m/U)."""
+    T = d = 16
+    rho, alpha, U = 1.5, 2.0, 8
+    K = np.zeros((1, 1, T, d), dtype=np.float32)
+    K[0, 0] = rho * np.eye(T, dtype=np.float32)
+    Q = np.zeros_like(K)
+    idx = np.zeros((1, T, U), dtype=np.int32)
+    want = np.zeros(T)
+    rng = np.random.default_rng(3)
+    for i in range(T):
+        p = (i * 5 + 1) % T
+        m = i % (U + 1)                     # 0..U occurrences of p
+        Q[0, 0, i] = alpha * K[0, 0, p]
+        others = [j for j in range(T) if j != p]
+        row = [p] * m + list(rng.choice(others, size=U - m))
+        rng.shuffle(row)
+        idx[0, i] = row
+        want[i] = 0.0 if m == 0 else (alpha * rho * rho / math.sqrt(d)) * (1.0 - m / U)
+    M = orc.measure(Q, K, idx, None, U_override=U)
+    np.testing.assert_allclose(M[0, 0], want, atol=1e-14)
+
+
+# ---- P6 / P7: relation to the exact measure (Eq. 10) --------------------------------------
+
+def test_full_sample_is_max_minus_mean_over_all_keys():
+    B, H, T, d = 1, 2, 20, 8
+    Q, K, V, _, lengths = _rand(B, H, T, d, 15, 1)
+    idx = np.tile(np.arange(T, dtype=np.int32), (B, T, 1))     # every key exactly once
+    M = orc.measure(Q, K, idx, lengths, U_override=T)
+    S = np.einsum("bhid,bhjd->bhij", Q.astype(np.float64), K.astype(np.float64)) / math.sqrt(d)
+    np.testing.assert_allclose(M, S.max(-1) - S.mean(-1), atol=1e-13)
+    # max <= LSE <= max + ln U  ==>  M~ <= M_exact <= M~ + ln U  on the same key multiset
+    Mx = orc.exact_measure(Q, K, lengths)
+    assert np.all(M <= Mx + 1e-12)
+    assert np.all(Mx <= M + math.log(T) + 1e-12)
+    lse = np.log(np.exp(S).sum(-1))
+    np.testing.assert_allclose(Mx, lse - S.mean(-1), atol=1e-12)
+
+
+# ---- P8: invariances -------------------------------------------------------------------
+
+def test_invariances():
+    B, H, T, d, c = 1, 2, 37, 16, 2.0
+    ncol = brute.n_count(c, T)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 16, ncol)
+    O, sel, M = orc.forward(Q, K, V, idx, lengths, c=c)
+    rng = np.random.default_rng(5)
+    # (i) order inside a sample row does not matter
+    idx2 = idx.copy()
+    for i in range(T):
+        rng.shuffle(idx2[0, i])
+    O2, sel2, M2 = orc.forward(Q, K, V, idx2, lengths, c=c)
+    np.testing.assert_allclose(M2, M, atol=1e-13)
+    np.testing.assert_array_equal(sel2, sel)
+    # (ii) permuting keys and values together (sample remapped) leaves everything unchanged
+    perm = rng.permutation(T)
+    inv = np.argsort(perm)
+    K3, V3 = K[:, :, perm], V[:, :, perm]
+    idx3 = inv[idx].astype(np.int32)
+    O3, sel3, M3 = orc.forward(Q, K3, V3, idx3, lengths, c=c)
+    np.testing.assert_allclose(M3, M, atol=1e-13)
+    np.testing.assert_array_equal(sel3, sel)
+    np.testing.assert_allclose(O3, O, atol=1e-12)
+    # (iii) one constant vector added to every key shifts all scores of a query equally
+    shift = rng.standard_normal(d).astype(np.float32)
+    K4 = (K.astype(np.float64) + shift).astype(np.float32)
+    O4, sel4, M4 = orc.forward(Q, K4, V, idx, lengths, c=c)
+    np.testing.assert_allclose(M4, M, atol=5e-5)      # float32 rounding of the shifted keys
+    np.testing.assert_allclose(O4, O, atol=5e-4)
+
+
+# ---- P9: linear in V; constant V -------------------------------------------------------
+
+def test_constant_value_rows_and_linearity():
+    B, H, T, d, c = 1, 2, 33, 8, 2.0
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 17, brute.n_count(c, T))
+    w = np.arange(1, d + 1, dtype=np.float32)
+    Vc = np.broadcast_to(w, V.shape).copy()
+    O, _, _ = orc.forward(Q, K, Vc, idx, lengths, c=c)
+    np.testing.assert_allclose(O, np.broadcast_to(w.astype(np.float64), O.shape), atol=1e-12)
+    V2 = np.random.default_rng(1).standard_normal(V.shape).astype(np.float32)
+    Oa, _, _ = orc.forward(Q, K, V, idx, lengths, c=c)
+    Ob, _, _ = orc.forward(Q, K, V2, idx, lengths, c=c)
+    Vs = (2.0 * V.astype(np.float64) + 0.5 * V2.astype(np.float64))
+    # 2V + V2/2 is exact in float32 only up to rounding; compare with that rounding in mind
+    Os, _, _ = orc.forward(Q, K, Vs.astype(np.float32), idx, lengths, c=c)
+    np.testing.assert_allclose(Os, 2.0 * Oa + 0.5 * Ob, atol=1e-5)
+
+
+# ---- P10: Q = 0 -> tie rule and uniform attention ----------------------------------------
+
+def test_zero_queries_pick_lowest_indices_and_output_mean():
+    B, H, T, d, c = 2, 2, 45, 8, 2.0
+    lengths = np.array([45, 20], dtype=np.int32)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 18, brute.n_count(c, T), lengths)
+    Q[:] = 0.0
+    O, sel, M = orc.forward(Q, K, V, idx, lengths, c=c)
+    assert np.all(M == 0.0)
+    vb = orc.mean_v(V, lengths)
+    for b in range(B):
+        L = int(lengths[b])
+        u = brute.n_count(c, L)
+        for h in range(H):
+            assert [int(x) for x in sel[b, h] if x >= 0] == list(range(u))
+            assert np.all(sel[b, h, u:] == -1)
+            np.testing.assert_allclose(O[b, h, :L], np.broadcast_to(vb[b, h], (L, d)), atol=1e-13)
+
+
+# ---- P11: planted spikes ---------------------------------------------------------------
+
+def test_planted_spikes_are_selected():
+    B, H, T, d, c = 1, 2, 96, 64, 3.0
+    u = brute.n_count(c, T)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 19, u)
+    Q *= 0.05                               # flat background
+    rng = np.random.default_rng(9)
+    planted = []
+    for h in range(H):
+        qs = np.sort(rng.choice(T, size=u, replace=False))
+        planted.append(list(int(x) for x in qs))
+    # the sample is shared by the heads, so plant the same key column for every query
+    for i in range(T):
+        idx[0, i, 0] = (i * 7 + 3) % T
+    for h in range(H):
+        for i in planted[h]:
+            Q[0, h, i] = 4.0 * K[0, h, idx[0, i, 0]]
+    _, sel, _ = orc.forward(Q, K, V, idx, lengths, c=c)
+    for h in range(H):
+        assert [int(x) for x in sel[0, h] if x >= 0] == planted[h]
+
+
+# ---- P12: padding --------------------------------------------------------------------------
+
+def test_padding_contents_and_padded_length_do_not_matter():
+    B, H, d, c = 2, 2, 16, 2.0
+    lengths = np.array([19, 26], dtype=np.int32)
+    T1, T2 = 26, 40
+    Q, K, V, idx, lengths = _rand(B, H, T1, d, 20, brute.n_count(c, T1), lengths)
+    O1, sel1, M1 = orc.forward(Q, K, V, idx, lengths, c=c)
+
+    def grow(x, fillv):
+        out = np.full((B, H, T2, d), fillv, dtype=np.float32)
+        for b in range(B):
+            out[b, :, :lengths[b]] = x[b, :, :lengths[b]]
+        return out
+
+    idx2 = np.zeros((B, T2, idx.shape[2]), dtype=np.int32)
+    idx2[:, :T1] = idx
+    O2, sel2, M2 = orc.forward(grow(Q, np.nan), grow(K, np.nan), grow(V, np.nan), idx2,
+                               lengths, c=c)
+    w1 = sel1.shape[-1]                     # u_max grows with the padded length; extra slots are -1
+    np.testing.assert_array_equal(sel2[..., :w1], sel1)
+    assert np.all(sel2[..., w1:] == -1)
+    for b in range(B):
+        L = int(lengths[b])
+        np.testing.assert_array_equal(O2[b, :, :L], O1[b, :, :L])
+        np.testing.assert_array_equal(M2[b, :, :L], M1[b, :, :L])
+        assert np.all(O2[b, :, L:] == 0.0)
+
+
+# ---- Sec. 4.4: a given index set is reused ------------------------------------------------
+
+def test_given_selection_is_used_as_is():
+    B, H, T, d, c = 1, 2, 30, 8, 2.0
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 21, brute.n_count(c, T))
+    sel_in = np.full((B, H, 4), -1, dtype=np.int32)
+    sel_in[0, 0, :3] = [2, 9, 17]
+    sel_in[0, 1, :4] = [0, 1, 28, 29]
+    O, sel, _ = orc.forward(Q, K, V, idx, lengths, c=c, sel_in=sel_in)
+    np.testing.assert_array_equal(sel, sel_in)
+    vb = orc.mean_v(V, lengths)
+    for h in range(H):
+        chosen = set(int(x) for x in sel_in[0, h] if x >= 0)
+        for i in range(T):
+            want = (brute.softmax_attention(Q[0, h, i], K[0, h], V[0, h]) if i in chosen
+                    else vb[0, h])
+            np.testing.assert_allclose(O[0, h, i], want, atol=1e-12)
+
+
+# ---- the seeded workloads themselves -----------------------------------------------------
+
+def test_workload_generator_is_deterministic_and_in_range():
+    w = wl.WORKLOADS["ragged_bf16"]
+    a = wl.make_inputs(w, 32, B=3)
+    b = wl.make_inputs(w, 32, B=3)
+    for k in a:
+        np.testing.assert_array_equal(a[k], b[k])
+    for bb in range(3):
+        L = int(a["lengths"][bb])
+        assert 40 <= L <= 500
+        assert a["sample_idx"][bb, :L].min() >= 0 and a["sample_idx"][bb, :L].max() < L
+        assert np.all(a["Q"][bb, :, L:] == 0)
+    # bf16 rounding: the low 16 bits of every value are zero, and rounding is to nearest even
+    assert np.all((a["Q"].view(np.uint32) & 0xFFFF) == 0)
+    x = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -20], dtype=np.float32)
+    r = wl.round_to_bf16(x)
+    np.testing.assert_array_equal(r, np.array([1.0, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7], dtype=np.float32))
+
+
+def test_peaky_queries_dominate_selection_on_tiny_workload():
+    """On the tiny workload most selected queries are peaky ones (they are what M~ detects)."""
+    w = wl.WORKLOADS["tiny_fp32"]
+    n = orc.count(w.c, w.T)
+    inp = wl.make_inputs(w, n)
+    _, sel, _ = orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c)
+    hits = sum(bool(inp["peaky"][0, h, i]) for h in range(w.H) for i in sel[0, h] if i >= 0)
+    total = int((sel >= 0).sum())
+    assert total == w.H * n
+    assert hits >= 0.3 * total      # 13 peaky of 128 per head; chance level would be ~10 %

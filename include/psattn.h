@@ -1,0 +1,173 @@
+/*
+ * psattn.h - C ABI of the prob-sparse multi-head self-attention forward library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The operation is the attention rule of arXiv 2106.09236, Sec. 3 ("Prob-Sparse
+ * Self-Attention"), applied independently to every (batch, head) unit:
+ *
+ *   (a) s_ij = q_i . k_j / sqrt(d) for the U sampled keys j of query i        (Eq. 11)
+ *   (b) M~_i = max_j s_ij - (1/U) sum_j s_ij                                   (Eq. 11)
+ *   (c) I_sparse = the u queries with the largest M~_i                         (Sec. 3.2)
+ *   (d) o_i = sum_j softmax_j(s_ij) v_j over all valid keys, for i in I_sparse (Eq. 7-8, Eq. 12)
+ *   (e) o_i = mean_j v_j over valid keys (or v_i, Eq. 12 as printed) otherwise (Sec. 3.1, Eq. 12)
+ *
+ * with U = u = n(c, len) = clamp(ceil(c ln len), 1, len) per sequence (Sec. 3.2:
+ * "L~ = r_sample ln L"), natural logarithm, evaluated on the host in double.
+ *
+ * Conventions common to every call
+ *   - All functions return an int status (PSATTN_OK == 0); none throws, aborts or
+ *     synchronises the device, except where stated.  All device work is enqueued on
+ *     the caller's stream (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - "device" pointers must be device memory of the GPU that was current when the
+ *     plan was created; "host" pointers are ordinary host memory.  The caller owns every
+ *     buffer.  After psattn_plan_create the library allocates nothing (exception:
+ *     psattn_plan_enable_host_io, which allocates staging buffers once).
+ *   - Q, K, V, O are [B][H][T_max][d_head] with d_head contiguous; the element strides of
+ *     the b, h and t axes are given in the descriptor (all zero = dense row-major).  Base
+ *     pointers must be 16-byte aligned and the strides multiples of 8 elements.
+ *     Element type: bf16 (PSATTN_BF16) or float (PSATTN_FP32); O has the input type.
+ *     Accumulation is always fp32.
+ *   - lengths: device int32 [B], valid length of each sequence (key-padding mask), or NULL
+ *     (every sequence has length T_max).  Values are clamped to [0, T_max] (status bit 1).
+ *     Rows of O at positions >= lengths[b] are written as zeros; Q, K, V there are never read.
+ *   - sample_idx: device int32, row (b, i) (or (b, h, i) with idx_per_head) holds the sampled
+ *     key positions of query i in its first U_b entries; row stride idx_cols elements.  Entries
+ *     must lie in [0, lengths[b]); others are clamped into range and status bit 0 is set.
+ *     A key that occurs twice counts twice in the mean of Eq. 11.
+ *   - sel_idx: device int32 [B][H][u_max], the selected query positions of each unit in
+ *     ascending order, padded with -1.  Equal M~ values are ordered by position (lower first).
+ *   - workspace: device scratch of at least psattn_workspace_bytes() bytes, 256-byte aligned.
+ *     Its first 256 bytes hold the status word and must be zero before the first call that
+ *     uses the buffer (psattn_read_status clears them again); the rest needs no initialisation.
+ *     Calls that share a workspace must be stream-ordered.
+ */
+#ifndef PSATTN_H_
+#define PSATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    PSATTN_OK = 0,
+    PSATTN_ERR_NULL = 1,                /* a required pointer is NULL */
+    PSATTN_ERR_BAD_DESC = 2,            /* a size, stride or enum in the descriptor is invalid */
+    PSATTN_ERR_UNSUPPORTED = 3,         /* valid request this build cannot run (e.g. d_head != 64) */
+    PSATTN_ERR_WORKSPACE_TOO_SMALL = 4,
+    PSATTN_ERR_MISALIGNED = 5,          /* a base pointer is not 16-byte aligned */
+    PSATTN_ERR_CUDA = 6,                /* a CUDA runtime call failed; see psattn_last_cuda_error */
+    PSATTN_ERR_NO_DEVICE = 7            /* no usable sm_100 device */
+};
+
+enum { PSATTN_BF16 = 0, PSATTN_FP32 = 1 };
+enum { PSATTN_FILL_MEAN_V = 0, PSATTN_FILL_OWN_V = 1 };
+enum { PSATTN_PATH_AUTO = 0, PSATTN_PATH_STAGED = 1, PSATTN_PATH_FUSED = 2 };
+
+/* bits of the device status word (psattn_read_status) */
+enum {
+    PSATTN_STATUS_IDX_CLAMPED = 1u,     /* a sample_idx / row index was out of range and clamped */
+    PSATTN_STATUS_LEN_CLAMPED = 2u,     /* a length was outside [0, T_max] and clamped */
+    PSATTN_STATUS_WAIT_EXPIRED = 4u     /* a bounded device-side wait gave up; results invalid */
+};
+
+typedef struct psattn_desc {
+    int32_t B, H, T_max, d_head;        /* d_head must be 64 */
+    int32_t dtype;                      /* PSATTN_BF16 | PSATTN_FP32 */
+    int32_t fill_mode;                  /* PSATTN_FILL_MEAN_V (default) | PSATTN_FILL_OWN_V */
+    int32_t u_override;                 /* > 0: select min(u_override, len) queries instead of n(c, len) */
+    int32_t U_override;                 /* > 0: use min(U_override, idx_cols) samples instead of n(c, len) */
+    int32_t idx_cols;                   /* row stride (elements) of sample_idx, >= largest U used */
+    int32_t idx_per_head;               /* 0: sample_idx is [B][T_max][idx_cols], shared by the heads;
+                                           1: [B][H][T_max][idx_cols] */
+    int32_t path;                       /* PSATTN_PATH_*: kernel schedule; AUTO picks per shape */
+    int32_t reserved;
+    double c;                           /* sampling factor of n(c, len) */
+    int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* b, h, t strides in elements; all 0 = dense */
+} psattn_desc_t;
+
+typedef struct psattn_plan psattn_plan_t;
+
+/* Library version (major * 1000 + minor). */
+int psattn_version(void);
+/* Static, NUL-terminated description of a status code. */
+const char *psattn_status_string(int status);
+/* Number of kernels this library has launched in this process so far (all plans, all streams). */
+unsigned long long psattn_launch_count(void);
+/* cudaError_t of the last failed runtime call seen through this plan (0 if none). */
+int psattn_last_cuda_error(const psattn_plan_t *plan);
+
+/* n(c, len) of Sec. 3.2 (host arithmetic in double): the sample size U and the number u of
+ * selected queries for a sequence of `len` valid positions.  Returns 0 for len <= 0. */
+int psattn_count(double c, int len);
+
+/* Validates the descriptor, builds the per-length tables u[len], U[len] (len = 0..T_max) on
+ * the host and uploads them, and records the current device.  *out is NULL on failure. */
+int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out);
+int psattn_plan_destroy(psattn_plan_t *plan);
+/* Largest u and U over len in [0, T_max]: the widths of sel_idx and the minimum idx_cols. */
+int psattn_plan_limits(const psattn_plan_t *plan, int32_t *u_max, int32_t *U_max);
+/* Bytes of device workspace every call below needs (the same size for all of them). */
+int psattn_workspace_bytes(const psattn_plan_t *plan, size_t *bytes);
+
+/* Steps (a)-(e) (Eq. 11, Sec. 3.2, Eq. 12).  All pointers device.  M_out (fp32
+ * [B][H][T_max], zero at padded positions) may be NULL. */
+int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                   const int32_t *lengths, const int32_t *sample_idx, void *O,
+                   int32_t *sel_idx, float *M_out, void *workspace, size_t workspace_bytes,
+                   void *stream);
+
+/* Steps (d)-(e) with a given index set (same layout as sel_idx; entries outside
+ * [0, lengths[b]) are ignored): the reuse of one layer's selection by the following layers
+ * (Sec. 4.4), and the random-selection ablation of Table 1. */
+int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q, const void *K,
+                                  const void *V, const int32_t *lengths,
+                                  const int32_t *sel_idx_in, void *O, void *workspace,
+                                  size_t workspace_bytes, void *stream);
+
+/* Steps (a)+(b) only (Eq. 11): M_out fp32 [B][H][T_max], zero at padded positions. */
+int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K, const int32_t *lengths,
+                   const int32_t *sample_idx, float *M_out, void *workspace,
+                   size_t workspace_bytes, void *stream);
+
+/* Step (c) only (Sec. 3.2): top-u positions of M (fp32 [B][H][T_max]) among i < lengths[b]. */
+int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
+                  int32_t *sel_idx, void *workspace, size_t workspace_bytes, void *stream);
+
+/* The fill value of step (e): vbar fp32 [B][H][d_head] = mean of V over valid keys (Sec. 3.1). */
+int psattn_mean_v(psattn_plan_t *plan, const void *V, const int32_t *lengths, float *vbar,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
+/* Step (d) only (Eq. 7-8) for listed rows: row_idx int32 [B][H][n_rows] (entries outside
+ * [0, lengths[b]) produce a zero row), out fp32 [B][H][n_rows][d_head]. n_rows <= u_max. */
+int psattn_attend_rows(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                       const int32_t *lengths, const int32_t *row_idx, int32_t n_rows,
+                       float *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Dense softmax attention (Eq. 6) for every valid query on the same layout: the comparator
+ * the sparse path is measured against.  Padded rows of O are zero. */
+int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                         const int32_t *lengths, void *O, void *workspace,
+                         size_t workspace_bytes, void *stream);
+
+/* Copies the device status word of `workspace` to *host_bits and clears it.  Synchronises
+ * `stream`. */
+int psattn_read_status(psattn_plan_t *plan, void *workspace, void *stream, uint32_t *host_bits);
+
+/* Host-buffer front end.  psattn_plan_enable_host_io allocates, once, device staging for
+ * Q, K, V, O, lengths, sample_idx, sel_idx and a workspace inside the plan.
+ * psattn_forward_host then copies the HOST arrays in (dense layout, descriptor strides
+ * ignored), runs psattn_forward, copies O and sel_idx back and synchronises the stream.
+ * lengths may be NULL.  Pinned host memory makes the copies asynchronous and fast; pageable
+ * memory works but is slower. */
+int psattn_plan_enable_host_io(psattn_plan_t *plan);
+int psattn_forward_host(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                        const int32_t *lengths, const int32_t *sample_idx, void *O,
+                        int32_t *sel_idx, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PSATTN_H_ */

@@ -1,0 +1,403 @@
+// C ABI of the library (see include/psattn.h): plan, validation, workspace layout and the
+// kernel schedules.  No kernel lives here.
+#include "../../include/psattn.h"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "psattn_launch.h"
+
+using namespace psattn;
+
+struct psattn_plan {
+    psattn_desc_t desc;
+    int device;
+    int u_max, U_max;
+    int n_chunks;                 // column-sum partials per unit
+    int n_splits;                 // key splits of the SIMT attention kernel
+    int *d_tables;                // device: u_tab[T+1] then U_tab[T+1]
+    int last_cuda_error;
+    // workspace layout (byte offsets)
+    size_t off_status, off_M, off_vpart, off_vbar, off_ml, off_acc, off_sel, ws_bytes;
+    // host-io staging (psattn_plan_enable_host_io)
+    bool host_io;
+    void *h_Q, *h_K, *h_V, *h_O, *h_ws;
+    int *h_len, *h_idx, *h_sel;
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+extern "C" int psattn_version(void) { return 1000; }
+
+extern "C" const char *psattn_status_string(int s) {
+    switch (s) {
+        case PSATTN_OK: return "ok";
+        case PSATTN_ERR_NULL: return "a required pointer is NULL";
+        case PSATTN_ERR_BAD_DESC: return "invalid descriptor or argument";
+        case PSATTN_ERR_UNSUPPORTED: return "unsupported configuration";
+        case PSATTN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case PSATTN_ERR_MISALIGNED: return "pointer not 16-byte aligned (workspace: 256-byte)";
+        case PSATTN_ERR_CUDA: return "CUDA runtime error";
+        case PSATTN_ERR_NO_DEVICE: return "no usable CUDA device";
+        default: return "unknown status";
+    }
+}
+
+extern "C" unsigned long long psattn_launch_count(void) { return launches_so_far(); }
+
+extern "C" int psattn_last_cuda_error(const psattn_plan_t *p) { return p ? p->last_cuda_error : 0; }
+
+extern "C" int psattn_count(double c, int len) {
+    if (len <= 0) return 0;
+    double x = std::ceil(c * std::log((double)len));
+    if (!(x >= 1.0)) x = 1.0;
+    if (x > (double)len) x = (double)len;
+    return (int)x;
+}
+
+static int cuda_fail(psattn_plan_t *p, cudaError_t e) {
+    if (p) p->last_cuda_error = (int)e;
+    return PSATTN_ERR_CUDA;
+}
+
+static bool strides_zero(const int64_t s[3]) { return s[0] == 0 && s[1] == 0 && s[2] == 0; }
+
+static int check_strides(int64_t s[3], const psattn_desc_t &d) {
+    if (strides_zero(s)) {
+        s[2] = d.d_head;
+        s[1] = (int64_t)d.T_max * d.d_head;
+        s[0] = (int64_t)d.H * d.T_max * d.d_head;
+        return PSATTN_OK;
+    }
+    for (int k = 0; k < 3; ++k)
+        if (s[k] < 0 || (s[k] % 8) != 0) return PSATTN_ERR_BAD_DESC;
+    if (s[2] < d.d_head) return PSATTN_ERR_BAD_DESC;
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!desc || !out) return PSATTN_ERR_NULL;
+    psattn_desc_t d = *desc;
+    if (d.B < 0 || d.H < 1 || d.T_max < 1 || d.B > (1 << 20) || d.H > 4096 || d.T_max > (1 << 20))
+        return PSATTN_ERR_BAD_DESC;
+    if ((long long)d.B * d.H > (1ll << 24)) return PSATTN_ERR_BAD_DESC;
+    if (d.dtype != PSATTN_BF16 && d.dtype != PSATTN_FP32) return PSATTN_ERR_BAD_DESC;
+    if (d.fill_mode != PSATTN_FILL_MEAN_V && d.fill_mode != PSATTN_FILL_OWN_V) return PSATTN_ERR_BAD_DESC;
+    if (d.path < PSATTN_PATH_AUTO || d.path > PSATTN_PATH_FUSED) return PSATTN_ERR_BAD_DESC;
+    if (d.u_override < 0 || d.U_override < 0 || d.idx_cols < 1) return PSATTN_ERR_BAD_DESC;
+    if (!(d.c > 0.0) || !std::isfinite(d.c)) return PSATTN_ERR_BAD_DESC;
+    if (d.d_head != kD) return PSATTN_ERR_UNSUPPORTED;
+    int rc;
+    if ((rc = check_strides(d.q_stride, d)) || (rc = check_strides(d.k_stride, d)) ||
+        (rc = check_strides(d.v_stride, d)) || (rc = check_strides(d.o_stride, d)))
+        return rc;
+
+    // per-length tables of Sec. 3.2's counts, in double on the host
+    std::vector<int> tab(2 * (size_t)(d.T_max + 1));
+    int u_max = 0, U_max = 0;
+    for (int len = 0; len <= d.T_max; ++len) {
+        int n = psattn_count(d.c, len);
+        int u = d.u_override > 0 ? (d.u_override < len ? d.u_override : len) : n;
+        int U = d.U_override > 0 ? (len > 0 ? d.U_override : 0) : n;
+        if (U > d.idx_cols) {
+            if (d.U_override > 0) U = d.idx_cols;
+            else return PSATTN_ERR_BAD_DESC;        // idx_cols narrower than the rule's U
+        }
+        tab[len] = u;
+        tab[d.T_max + 1 + len] = U;
+        if (u > u_max) u_max = u;
+        if (U > U_max) U_max = U;
+    }
+    if (u_max < 1) u_max = 1;
+
+    int dev = 0, ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) { cudaGetLastError(); return PSATTN_ERR_NO_DEVICE; }
+    if (cudaGetDevice(&dev) != cudaSuccess) return PSATTN_ERR_NO_DEVICE;
+    int major = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return PSATTN_ERR_NO_DEVICE;
+
+    psattn_plan_t *p = new (std::nothrow) psattn_plan_t();
+    if (!p) return PSATTN_ERR_CUDA;
+    std::memset(p, 0, sizeof(*p));
+    p->desc = d;
+    p->device = dev;
+    p->u_max = u_max;
+    p->U_max = U_max;
+    p->n_chunks = (d.T_max + kColsumRows - 1) / kColsumRows;
+    p->n_splits = (d.T_max + kSplitKeys - 1) / kSplitKeys;
+    cudaError_t e = cudaMalloc((void **)&p->d_tables, tab.size() * sizeof(int));
+    if (e != cudaSuccess) { delete p; return PSATTN_ERR_CUDA; }
+    e = cudaMemcpy(p->d_tables, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(p->d_tables); delete p; return PSATTN_ERR_CUDA; }
+
+    const size_t units = (size_t)d.B * d.H;
+    size_t off = 0;
+    p->off_status = off; off = align_up(off + 256, 256);
+    p->off_M = off;      off = align_up(off + units * d.T_max * sizeof(float), 256);
+    p->off_vpart = off;  off = align_up(off + units * p->n_chunks * kD * sizeof(float), 256);
+    p->off_vbar = off;   off = align_up(off + units * kD * sizeof(float), 256);
+    p->off_ml = off;     off = align_up(off + units * u_max * p->n_splits * 2 * sizeof(float), 256);
+    p->off_acc = off;    off = align_up(off + units * u_max * p->n_splits * kD * sizeof(float), 256);
+    p->off_sel = off;    off = align_up(off + units * u_max * sizeof(int), 256);
+    p->ws_bytes = off;
+    *out = p;
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_plan_destroy(psattn_plan_t *p) {
+    if (!p) return PSATTN_ERR_NULL;
+    cudaFree(p->d_tables);
+    if (p->host_io) {
+        cudaFree(p->h_Q); cudaFree(p->h_K); cudaFree(p->h_V); cudaFree(p->h_O); cudaFree(p->h_ws);
+        cudaFree(p->h_len); cudaFree(p->h_idx); cudaFree(p->h_sel);
+    }
+    delete p;
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_plan_limits(const psattn_plan_t *p, int32_t *u_max, int32_t *U_max) {
+    if (!p) return PSATTN_ERR_NULL;
+    if (u_max) *u_max = p->u_max;
+    if (U_max) *U_max = p->U_max;
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_workspace_bytes(const psattn_plan_t *p, size_t *bytes) {
+    if (!p || !bytes) return PSATTN_ERR_NULL;
+    *bytes = p->ws_bytes;
+    return PSATTN_OK;
+}
+
+// ---- helpers ---------------------------------------------------------------------------
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_ws(const psattn_plan_t *p, const void *ws, size_t bytes) {
+    if (!ws) return PSATTN_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PSATTN_ERR_MISALIGNED;
+    if (bytes < p->ws_bytes) return PSATTN_ERR_WORKSPACE_TOO_SMALL;
+    return PSATTN_OK;
+}
+
+static Geom make_geom(const psattn_plan_t *p, const int32_t *lengths, void *ws) {
+    Geom g;
+    const psattn_desc_t &d = p->desc;
+    g.B = d.B; g.H = d.H; g.T = d.T_max;
+    g.idx_cols = d.idx_cols; g.idx_per_head = d.idx_per_head;
+    g.u_max = p->u_max;
+    for (int k = 0; k < 3; ++k) {
+        g.qs[k] = d.q_stride[k]; g.ks[k] = d.k_stride[k];
+        g.vs[k] = d.v_stride[k]; g.os[k] = d.o_stride[k];
+    }
+    g.lengths = lengths;
+    g.u_tab = p->d_tables;
+    g.U_tab = p->d_tables + d.T_max + 1;
+    g.status = reinterpret_cast<unsigned *>(static_cast<char *>(ws) + p->off_status);
+    return g;
+}
+
+template <typename T>
+static T *ws_at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast<char *>(ws) + off); }
+
+#define PSATTN_CU(expr)                                         \
+    do {                                                        \
+        cudaError_t e__ = (expr);                               \
+        if (e__ != cudaSuccess) return cuda_fail(plan, e__);    \
+    } while (0)
+
+// Steps (d)+(e) for a selection that already sits in `sel` (device) with vbar in the workspace.
+static int run_attend_and_fill(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K,
+                               const void *V, const int *sel, void *O, void *ws, cudaStream_t st) {
+    const psattn_desc_t &d = plan->desc;
+    PSATTN_CU(launch_fill(d.dtype, g, V, sel, ws_at<float>(ws, plan->off_vbar), O,
+                          d.fill_mode == PSATTN_FILL_OWN_V, st));
+    PSATTN_CU(launch_attend_simt(d.dtype, 0, g, Q, K, V, sel, plan->u_max, plan->u_max,
+                                 plan->n_splits, kSplitKeys, ws_at<float>(ws, plan->off_ml),
+                                 ws_at<float>(ws, plan->off_acc), O, 0, 0, 1, st));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                              const int32_t *lengths, const int32_t *sample_idx, void *O,
+                              int32_t *sel_idx, float *M_out, void *workspace,
+                              size_t workspace_bytes, void *stream) {
+    if (!plan || !Q || !K || !V || !sample_idx || !O || !sel_idx) return PSATTN_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const psattn_desc_t &d = plan->desc;
+    Geom g = make_geom(plan, lengths, workspace);
+    float *M = M_out ? M_out : ws_at<float>(workspace, plan->off_M);
+    PSATTN_CU(launch_measure(d.dtype, g, Q, K, sample_idx, M, st));
+    PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
+    PSATTN_CU(launch_select(g, M, sel_idx, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks,
+                            ws_at<float>(workspace, plan->off_vbar), st));
+    return run_attend_and_fill(plan, g, Q, K, V, sel_idx, O, workspace, st);
+}
+
+extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q, const void *K,
+                                             const void *V, const int32_t *lengths,
+                                             const int32_t *sel_idx_in, void *O, void *workspace,
+                                             size_t workspace_bytes, void *stream) {
+    if (!plan || !Q || !K || !V || !sel_idx_in || !O) return PSATTN_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const psattn_desc_t &d = plan->desc;
+    Geom g = make_geom(plan, lengths, workspace);
+    // mean(V): column sums, then the finishing part of the select kernel is not needed; use a
+    // select launch with u forced to nothing?  Simpler and exact: the same two kernels.
+    PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
+    PSATTN_CU(launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart),
+                            plan->n_chunks, ws_at<float>(workspace, plan->off_vbar), st));
+    return run_attend_and_fill(plan, g, Q, K, V, sel_idx_in, O, workspace, st);
+}
+
+extern "C" int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K,
+                              const int32_t *lengths, const int32_t *sample_idx, float *M_out,
+                              void *workspace, size_t workspace_bytes, void *stream) {
+    if (!plan || !Q || !K || !sample_idx || !M_out) return PSATTN_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    Geom g = make_geom(plan, lengths, workspace);
+    PSATTN_CU(launch_measure(plan->desc.dtype, g, Q, K, sample_idx, M_out, static_cast<cudaStream_t>(stream)));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
+                             int32_t *sel_idx, void *workspace, size_t workspace_bytes,
+                             void *stream) {
+    if (!plan || !M || !sel_idx) return PSATTN_ERR_NULL;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    Geom g = make_geom(plan, lengths, workspace);
+    PSATTN_CU(launch_select(g, M, sel_idx, nullptr, 0, nullptr, static_cast<cudaStream_t>(stream)));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_mean_v(psattn_plan_t *plan, const void *V, const int32_t *lengths,
+                             float *vbar, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!plan || !V || !vbar) return PSATTN_ERR_NULL;
+    if (!aligned16(V)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    Geom g = make_geom(plan, lengths, workspace);
+    PSATTN_CU(launch_colsum(plan->desc.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
+    PSATTN_CU(launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, vbar, st));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_attend_rows(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                                  const int32_t *lengths, const int32_t *row_idx, int32_t n_rows,
+                                  float *out, void *workspace, size_t workspace_bytes,
+                                  void *stream) {
+    if (!plan || !Q || !K || !V || !row_idx || !out) return PSATTN_ERR_NULL;
+    if (n_rows < 0 || n_rows > plan->u_max) return PSATTN_ERR_BAD_DESC;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    if (n_rows == 0) return PSATTN_OK;
+    Geom g = make_geom(plan, lengths, workspace);
+    PSATTN_CU(launch_attend_simt(plan->desc.dtype, 1, g, Q, K, V, row_idx, n_rows, n_rows,
+                                 plan->n_splits, kSplitKeys, ws_at<float>(workspace, plan->off_ml),
+                                 ws_at<float>(workspace, plan->off_acc), out,
+                                 (long long)n_rows * kD, kD, 0, static_cast<cudaStream_t>(stream)));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const void *K,
+                                    const void *V, const int32_t *lengths, void *O,
+                                    void *workspace, size_t workspace_bytes, void *stream) {
+    if (!plan || !Q || !K || !V || !O) return PSATTN_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const psattn_desc_t &d = plan->desc;
+    Geom g = make_geom(plan, lengths, workspace);
+    // zero rows at padded positions: a fill with an empty selection and a zero "mean" would
+    // also overwrite valid rows, so fill first (mean value irrelevant) and let attention
+    // overwrite every valid row.
+    int *sel = ws_at<int>(workspace, plan->off_sel);
+    PSATTN_CU(cudaMemsetAsync(sel, 0xff, (size_t)d.B * d.H * plan->u_max * sizeof(int), st));
+    PSATTN_CU(cudaMemsetAsync(ws_at<float>(workspace, plan->off_vbar), 0, (size_t)d.B * d.H * kD * sizeof(float), st));
+    PSATTN_CU(launch_fill(d.dtype, g, V, sel, ws_at<float>(workspace, plan->off_vbar), O, 0, st));
+    PSATTN_CU(launch_attend_simt(d.dtype, 0, g, Q, K, V, nullptr, d.T_max, 0, 1, d.T_max, nullptr,
+                                 nullptr, O, 0, 0, 1, st));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_read_status(psattn_plan_t *plan, void *workspace, void *stream,
+                                  uint32_t *host_bits) {
+    if (!plan || !workspace || !host_bits) return PSATTN_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned *w = ws_at<unsigned>(workspace, plan->off_status);
+    PSATTN_CU(cudaMemcpyAsync(host_bits, w, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
+    PSATTN_CU(cudaMemsetAsync(w, 0, sizeof(unsigned), st));
+    PSATTN_CU(cudaStreamSynchronize(st));
+    return PSATTN_OK;
+}
+
+// ---- host-buffer front end ------------------------------------------------------------------
+extern "C" int psattn_plan_enable_host_io(psattn_plan_t *plan) {
+    if (!plan) return PSATTN_ERR_NULL;
+    if (plan->host_io) return PSATTN_OK;
+    const psattn_desc_t &d = plan->desc;
+    const size_t es = d.dtype == PSATTN_BF16 ? 2 : 4;
+    const size_t n = (size_t)d.B * d.H * d.T_max * kD * es;
+    const size_t nidx = (size_t)d.B * (d.idx_per_head ? d.H : 1) * d.T_max * d.idx_cols * sizeof(int);
+    void **bufs[] = {&plan->h_Q, &plan->h_K, &plan->h_V, &plan->h_O, &plan->h_ws,
+                     (void **)&plan->h_len, (void **)&plan->h_idx, (void **)&plan->h_sel};
+    const size_t sizes[] = {n, n, n, n, plan->ws_bytes, (size_t)d.B * sizeof(int) + 16, nidx + 16,
+                            (size_t)d.B * d.H * plan->u_max * sizeof(int) + 16};
+    for (int k = 0; k < 8; ++k) {
+        cudaError_t e = cudaMalloc(bufs[k], sizes[k] ? sizes[k] : 16);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < k; ++j) { cudaFree(*bufs[j]); *bufs[j] = nullptr; }
+            return cuda_fail(plan, e);
+        }
+    }
+    PSATTN_CU(cudaMemset(plan->h_ws, 0, 256));
+    plan->host_io = true;
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_forward_host(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
+                                   const int32_t *lengths, const int32_t *sample_idx, void *O,
+                                   int32_t *sel_idx, void *stream) {
+    if (!plan || !Q || !K || !V || !sample_idx || !O || !sel_idx) return PSATTN_ERR_NULL;
+    if (!plan->host_io) return PSATTN_ERR_BAD_DESC;
+    psattn_desc_t &d = plan->desc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t es = d.dtype == PSATTN_BF16 ? 2 : 4;
+    const size_t n = (size_t)d.B * d.H * d.T_max * kD * es;
+    const size_t nidx = (size_t)d.B * (d.idx_per_head ? d.H : 1) * d.T_max * d.idx_cols * sizeof(int);
+    const size_t nsel = (size_t)d.B * d.H * plan->u_max * sizeof(int);
+    PSATTN_CU(cudaMemcpyAsync(plan->h_Q, Q, n, cudaMemcpyHostToDevice, st));
+    PSATTN_CU(cudaMemcpyAsync(plan->h_K, K, n, cudaMemcpyHostToDevice, st));
+    PSATTN_CU(cudaMemcpyAsync(plan->h_V, V, n, cudaMemcpyHostToDevice, st));
+    PSATTN_CU(cudaMemcpyAsync(plan->h_idx, sample_idx, nidx, cudaMemcpyHostToDevice, st));
+    if (lengths) PSATTN_CU(cudaMemcpyAsync(plan->h_len, lengths, (size_t)d.B * sizeof(int), cudaMemcpyHostToDevice, st));
+    // the staging buffers are dense: run with dense strides whatever the descriptor says
+    psattn_desc_t saved = d;
+    std::memset(d.q_stride, 0, sizeof(d.q_stride)); std::memset(d.k_stride, 0, sizeof(d.k_stride));
+    std::memset(d.v_stride, 0, sizeof(d.v_stride)); std::memset(d.o_stride, 0, sizeof(d.o_stride));
+    check_strides(d.q_stride, d); check_strides(d.k_stride, d);
+    check_strides(d.v_stride, d); check_strides(d.o_stride, d);
+    int rc = psattn_forward(plan, plan->h_Q, plan->h_K, plan->h_V, lengths ? plan->h_len : nullptr,
+                            plan->h_idx, plan->h_O, plan->h_sel, nullptr, plan->h_ws,
+                            plan->ws_bytes, stream);
+    d = saved;
+    if (rc) return rc;
+    PSATTN_CU(cudaMemcpyAsync(O, plan->h_O, n, cudaMemcpyDeviceToHost, st));
+    PSATTN_CU(cudaMemcpyAsync(sel_idx, plan->h_sel, nsel, cudaMemcpyDeviceToHost, st));
+    PSATTN_CU(cudaStreamSynchronize(st));
+    return PSATTN_OK;
+}

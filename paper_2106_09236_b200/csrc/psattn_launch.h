@@ -1,0 +1,33 @@
+// Host-callable launchers of the kernels; shared by the translation units of the library.
+#pragma once
+#include "psattn_common.cuh"
+
+namespace psattn {
+
+constexpr int kColsumRows = 256;      // rows of V per column-sum partial
+constexpr int kFillRows = 128;        // rows of O per fill block
+constexpr int kSelectThreads = 512;
+constexpr int kSplitKeys = 1024;      // keys per split of the SIMT attention kernel
+
+// Every kernel launch of the library is counted (process-wide).
+void note_launch(int n = 1);
+unsigned long long launches_so_far();
+
+cudaError_t launch_measure(int dtype, const Geom &g, const void *Q, const void *K, const int *sidx,
+                           float *M, cudaStream_t st);
+cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, int n_chunks,
+                          cudaStream_t st);
+cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,
+                          float *vbar, cudaStream_t st);
+// rows == nullptr: the row list is the identity (row r is position r).
+// out_by_position: write the finished row at its position in O (element type of the inputs,
+// strides g.os); otherwise at slot r of `out` with the given unit / row strides.
+cudaError_t launch_attend_simt(int dtype, int out_fp32, const Geom &g, const void *Q, const void *K,
+                               const void *V, const int *rows, int n_rows, int rows_stride,
+                               int n_splits, int split_keys, float *part_ml, float *part_acc,
+                               void *out, long long out_unit_stride, long long out_row_stride,
+                               int out_by_position, cudaStream_t st);
+cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
+                        void *O, int own_v, cudaStream_t st);
+
+}  // namespace psattn

@@ -1,0 +1,461 @@
+// Staged (one kernel per step) schedule of prob-sparse attention: plain SIMT kernels that
+// run for any T_max, both element types, and serve the per-step entry points.
+//   measure  : steps (a)+(b), Eq. 11           select : step (c), Sec. 3.2
+//   colsum   : partial column sums of V        fill   : step (e), Eq. 12 else-branch
+//   attend   : step (d), Eq. 7-8, flash-decoding form with one key per lane
+#include "psattn_launch.h"
+
+#include <atomic>
+
+namespace psattn {
+
+// ---------------------------------------------------------------------------------------
+// Steps (a)+(b): one warp per query.  The warp is four groups of eight lanes; a group
+// reads one sampled key row per step (lane `sub` holds columns 8*sub..8*sub+7 of q and of
+// the key), reduces the dot product over its eight lanes and keeps a MeasureState.
+// ---------------------------------------------------------------------------------------
+template <typename DT>
+__global__ void __launch_bounds__(256) k_measure(Geom g, const DT *__restrict__ Q,
+                                                 const DT *__restrict__ K,
+                                                 const int *__restrict__ sidx,
+                                                 float *__restrict__ M) {
+    const int lane = threadIdx.x & 31, sub = lane & 7, grp = lane >> 3;
+    const long long w = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long total = (long long)g.B * g.H * g.T;
+    if (w >= total) return;
+    const int i = (int)(w % g.T);
+    const int unit = (int)(w / g.T);
+    const int b = unit / g.H, h = unit % g.H;
+    const int L = seq_len(g, b);
+    if (i >= L) { if (lane == 0) M[w] = 0.f; return; }
+    const int U = min(g.U_tab[L], g.idx_cols);
+
+    float q[8];
+    load8(Q + unit_off(g.qs, b, h) + (long long)i * g.qs[2], sub, q);
+    const DT *Ku = K + unit_off(g.ks, b, h);
+    const int *row = sidx + ((g.idx_per_head ? (long long)unit : (long long)b) * g.T + i) * g.idx_cols;
+
+    MeasureState st = measure_init();
+    for (int base = 0; base < U; base += 32) {
+        int my = 0;
+        if (base + lane < U) {
+            my = __ldg(row + base + lane);
+            if (my < 0 || my >= L) { atomicOr(g.status, kStatusIdxClamped); my = my < 0 ? 0 : L - 1; }
+        }
+        const int steps = (min(32, U - base) + 3) >> 2;
+        for (int s = 0; s < steps; ++s) {
+            const int src = s * 4 + grp;
+            const int key = __shfl_sync(0xffffffffu, my, src);
+            const bool active = base + src < U;
+            float kk[8];
+            float part = 0.f;
+            if (active) {
+                load8(Ku + (long long)key * g.ks[2], sub, kk);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) part = fmaf(q[t], kk[t], part);
+            }
+            part += __shfl_xor_sync(0xffffffffu, part, 1);
+            part += __shfl_xor_sync(0xffffffffu, part, 2);
+            part += __shfl_xor_sync(0xffffffffu, part, 4);
+            if (active) measure_push(st, part * kScale);
+        }
+    }
+#pragma unroll
+    for (int o = 8; o <= 16; o <<= 1) {
+        MeasureState other;
+        other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+        other.D = __shfl_xor_sync(0xffffffffu, st.D, o);
+        other.n = __shfl_xor_sync(0xffffffffu, st.n, o);
+        // merge in a fixed (lower group first) order so that all lanes agree bit for bit
+        st = (lane & o) ? measure_merge(other, st) : measure_merge(st, other);
+    }
+    if (lane == 0) M[w] = U > 0 ? st.D / (float)U : 0.f;
+}
+
+// ---------------------------------------------------------------------------------------
+// Column sums of V over blocks of kColsumRows valid rows: part[unit][chunk][64].
+// ---------------------------------------------------------------------------------------
+template <typename DT>
+__global__ void __launch_bounds__(256) k_colsum(Geom g, const DT *__restrict__ V,
+                                                float *__restrict__ part, int n_chunks) {
+    __shared__ float red[32][kD + 1];
+    const int unit = blockIdx.x, chunk = blockIdx.y;
+    const int b = unit / g.H, h = unit % g.H;
+    const int L = seq_len(g, b);
+    const int sub = threadIdx.x & 7, r0 = threadIdx.x >> 3;
+    const int lo = chunk * kColsumRows, hi = min(L, lo + kColsumRows);
+    const DT *Vu = V + unit_off(g.vs, b, h);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int r = lo + r0; r < hi; r += 32) {
+        float v[8];
+        load8(Vu + (long long)r * g.vs[2], sub, v);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) acc[t] += v[t];
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) red[r0][sub * 8 + t] = acc[t];
+    __syncthreads();
+    if (threadIdx.x < kD) {
+        float s = 0.f;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) s += red[r][threadIdx.x];
+        part[((long long)unit * n_chunks + chunk) * kD + threadIdx.x] = s;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Step (c): one block per unit.  Four 8-bit radix passes over order-preserving keys find
+// the u-th largest value tau; the result is every position with key > tau plus the first
+// (in position order) positions with key == tau, written in ascending position order.
+// The same block finishes mean(V) from the column-sum partials.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot, int &total) {
+    // blockDim.x == kSelectThreads (a multiple of 32, <= 1024); v in {0,1,...}
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    int x = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+    }
+    if (lane == 31) warp_tot[wid] = x;
+    __syncthreads();
+    int before = 0, tot = 0;
+    for (int k = 0; k < nw; ++k) {
+        int t = warp_tot[k];
+        if (k < wid) before += t;
+        tot += t;
+    }
+    __syncthreads();
+    total = tot;
+    return before + x - v;
+}
+
+__global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *__restrict__ M,
+                                                           int *__restrict__ sel,
+                                                           const float *__restrict__ vpart,
+                                                           int n_chunks, float *__restrict__ vbar) {
+    __shared__ int hist[256];
+    __shared__ int warp_tot[32];
+    __shared__ unsigned s_prefix;
+    __shared__ int s_remaining;
+    const int unit = blockIdx.x;
+    const int b = unit / g.H;
+    const int L = seq_len(g, b);
+    const int u = min(min(g.u_tab[L], g.u_max), L);
+    const float *Mu = M + (long long)unit * g.T;
+    int *out = sel + (long long)unit * g.u_max;
+
+    if (vbar != nullptr && threadIdx.x < kD) {
+        float s = 0.f;
+        for (int c = 0; c < n_chunks; ++c) s += vpart[((long long)unit * n_chunks + c) * kD + threadIdx.x];
+        vbar[(long long)unit * kD + threadIdx.x] = L > 0 ? s / (float)L : 0.f;
+    }
+    if (M == nullptr) return;                  // mean(V) only
+    if (u <= 0) {
+        for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) out[r] = -1;
+        return;
+    }
+    if (threadIdx.x == 0) { s_prefix = 0u; s_remaining = u; }
+    unsigned known = 0u;                       // mask of the key bits fixed so far
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        for (int t = threadIdx.x; t < 256; t += blockDim.x) hist[t] = 0;
+        __syncthreads();
+        const unsigned prefix = s_prefix;
+        for (int i = threadIdx.x; i < L; i += blockDim.x) {
+            unsigned k = float_key(Mu[i]);
+            if (((k ^ prefix) & known) == 0u) atomicAdd(&hist[(k >> shift) & 255u], 1);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int rem = s_remaining, bin = 255;
+            for (; bin > 0; --bin) {
+                if (hist[bin] >= rem) break;
+                rem -= hist[bin];
+            }
+            s_prefix = prefix | ((unsigned)bin << shift);
+            s_remaining = rem;
+        }
+        known |= 0xffu << shift;
+        __syncthreads();
+    }
+    const unsigned tau = s_prefix;
+    const int need_eq = s_remaining;           // how many of the positions with key == tau to take
+    int eq_seen = 0, written = 0;
+    for (int base = 0; base < L; base += blockDim.x) {
+        const int i = base + threadIdx.x;
+        unsigned k = 0u;
+        const bool valid = i < L;
+        if (valid) k = float_key(Mu[i]);
+        const int is_eq = valid && k == tau;
+        int tot_eq, tot_take;
+        const int eq_rank = eq_seen + block_exclusive_scan(is_eq, warp_tot, tot_eq);
+        const int take = valid && (k > tau || (is_eq && eq_rank < need_eq));
+        const int pos = written + block_exclusive_scan(take, warp_tot, tot_take);
+        if (take && pos < g.u_max) out[pos] = i;
+        eq_seen += tot_eq;
+        written += tot_take;
+    }
+    for (int r = written + threadIdx.x; r < g.u_max; r += blockDim.x) out[r] = -1;
+}
+
+// ---------------------------------------------------------------------------------------
+// Step (d), SIMT form: one warp per (unit, listed row, key split).  Lane l owns keys
+// lo + l, lo + l + 32, ... and keeps its own online-softmax state (m, l, acc[64]) in base-2
+// exponent form; the 32 states are merged at the end.  With one split the row is finished
+// here; otherwise (m, l, acc) goes to the workspace for k_attend_combine.
+// ---------------------------------------------------------------------------------------
+template <typename DT>
+__device__ __forceinline__ void load_row64(const DT *row, float out[kD]) {
+#pragma unroll
+    for (int s = 0; s < 8; ++s) load8(row, s, out + 8 * s);
+}
+
+template <typename DT, typename OT>
+__global__ void __launch_bounds__(128) k_attend(Geom g, const DT *__restrict__ Q,
+                                                const DT *__restrict__ K,
+                                                const DT *__restrict__ V,
+                                                const int *__restrict__ rows, int n_rows,
+                                                int rows_stride, int n_splits, int split_keys,
+                                                float *__restrict__ part_ml,
+                                                float *__restrict__ part_acc,
+                                                OT *__restrict__ out, long long out_unit_stride,
+                                                long long out_row_stride, int out_by_position) {
+    const int lane = threadIdx.x & 31;
+    const long long w = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const long long total = (long long)g.B * g.H * n_rows * n_splits;
+    if (w >= total) return;
+    const int split = (int)(w % n_splits);
+    const int r = (int)((w / n_splits) % n_rows);
+    const int unit = (int)(w / ((long long)n_splits * n_rows));
+    const int b = unit / g.H, h = unit % g.H;
+    const int L = seq_len(g, b);
+    const int i = rows ? rows[(long long)unit * rows_stride + r] : r;
+    const bool row_ok = i >= 0 && i < L;
+    // where the finished row goes: at its position i of O, or at its slot r of a row-list output
+    OT *dst = nullptr;
+    if (out_by_position) { if (row_ok) dst = out + unit_off(g.os, b, h) + (long long)i * g.os[2]; }
+    else dst = out + (long long)unit * out_unit_stride + (long long)r * out_row_stride;
+
+    float m = -INFINITY, l = 0.f;
+    float acc[kD];
+#pragma unroll
+    for (int c = 0; c < kD; ++c) acc[c] = 0.f;
+    if (row_ok) {
+        float q[kD];
+        load_row64(Q + unit_off(g.qs, b, h) + (long long)i * g.qs[2], q);
+        const DT *Ku = K + unit_off(g.ks, b, h);
+        const DT *Vu = V + unit_off(g.vs, b, h);
+        const int lo = split * split_keys, hi = min(L, lo + split_keys);
+        for (int j = lo + lane; j < hi; j += 32) {
+            float x[kD];
+            load_row64(Ku + (long long)j * g.ks[2], x);
+            float s = 0.f;
+#pragma unroll
+            for (int c = 0; c < kD; ++c) s = fmaf(q[c], x[c], s);
+            s *= kScale * kLog2e;
+            if (s > m) {
+                const float f = exp2f(m - s);          // 0 on the first key (m = -inf)
+                l *= f;
+#pragma unroll
+                for (int c = 0; c < kD; ++c) acc[c] *= f;
+                m = s;
+            }
+            const float p = exp2f(s - m);
+            l += p;
+            load_row64(Vu + (long long)j * g.vs[2], x);
+#pragma unroll
+            for (int c = 0; c < kD; ++c) acc[c] = fmaf(p, x[c], acc[c]);
+        }
+    }
+    // merge the 32 lane states
+    float mw = m;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(0xffffffffu, mw, o));
+    const float f = (l > 0.f) ? exp2f(m - mw) : 0.f;
+    float lw = l * f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) lw += __shfl_xor_sync(0xffffffffu, lw, o);
+    float mine[2] = {0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < kD; ++c) {
+        float v = acc[c] * f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == (c & 31)) mine[c >> 5] = v;
+    }
+    if (n_splits == 1) {
+        if (dst) {
+            const float inv = lw > 0.f ? 1.f / lw : 0.f;
+            dst[lane] = (OT)(mine[0] * inv);
+            dst[lane + 32] = (OT)(mine[1] * inv);
+        }
+    } else {
+        const long long slot = ((long long)unit * n_rows + r) * n_splits + split;
+        if (lane == 0) { part_ml[2 * slot] = mw; part_ml[2 * slot + 1] = lw; }
+        part_acc[slot * kD + lane] = mine[0];
+        part_acc[slot * kD + lane + 32] = mine[1];
+    }
+}
+
+// Merge of the key splits of one row: 64 threads per row.
+template <typename OT>
+__global__ void __launch_bounds__(256) k_attend_combine(Geom g, const int *__restrict__ rows,
+                                                        int n_rows, int rows_stride, int n_splits,
+                                                        const float *__restrict__ part_ml,
+                                                        const float *__restrict__ part_acc,
+                                                        OT *__restrict__ out,
+                                                        long long out_unit_stride,
+                                                        long long out_row_stride,
+                                                        int out_by_position) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long rowid = t / kD;
+    const int c = (int)(t % kD);
+    if (rowid >= (long long)g.B * g.H * n_rows) return;
+    const int r = (int)(rowid % n_rows);
+    const int unit = (int)(rowid / n_rows);
+    const int b = unit / g.H, h = unit % g.H;
+    const int L = seq_len(g, b);
+    const int i = rows ? rows[(long long)unit * rows_stride + r] : r;
+    const bool row_ok = i >= 0 && i < L;
+    OT *dst;
+    if (out_by_position) {
+        if (!row_ok) return;
+        dst = out + unit_off(g.os, b, h) + (long long)i * g.os[2];
+    } else {
+        dst = out + (long long)unit * out_unit_stride + (long long)r * out_row_stride;
+    }
+    const long long slot0 = rowid * n_splits;
+    float mw = -INFINITY;
+    for (int s = 0; s < n_splits; ++s) mw = fmaxf(mw, part_ml[2 * (slot0 + s)]);
+    float lw = 0.f, a = 0.f;
+    for (int s = 0; s < n_splits; ++s) {
+        const float ls = part_ml[2 * (slot0 + s) + 1];
+        const float f = ls > 0.f ? exp2f(part_ml[2 * (slot0 + s)] - mw) : 0.f;
+        lw += ls * f;
+        a += part_acc[(slot0 + s) * kD + c] * f;
+    }
+    dst[c] = (OT)(lw > 0.f ? a / lw : 0.f);
+}
+
+// ---------------------------------------------------------------------------------------
+// Step (e): every valid, non-selected row of O receives mean(V) (or its own value row);
+// padded rows receive zeros; selected rows are left to step (d).  One block covers
+// kFillRows rows of one unit.
+// ---------------------------------------------------------------------------------------
+template <typename DT>
+__global__ void __launch_bounds__(256) k_fill(Geom g, const DT *__restrict__ V,
+                                              const int *__restrict__ sel,
+                                              const float *__restrict__ vbar, DT *__restrict__ O,
+                                              int own_v) {
+    __shared__ unsigned char chosen[kFillRows];
+    const int unit = blockIdx.x;
+    const int b = unit / g.H, h = unit % g.H;
+    const int L = seq_len(g, b);
+    const int lo = blockIdx.y * kFillRows;
+    for (int t = threadIdx.x; t < kFillRows; t += blockDim.x) chosen[t] = 0;
+    __syncthreads();
+    for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) {
+        const int i = sel[(long long)unit * g.u_max + r];
+        if (i >= lo && i < lo + kFillRows && i < L) chosen[i - lo] = 1;
+    }
+    __syncthreads();
+    const int sub = threadIdx.x & 7, r0 = threadIdx.x >> 3;
+    float mean8[8], zero8[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { mean8[t] = vbar[(long long)unit * kD + sub * 8 + t]; zero8[t] = 0.f; }
+    DT *Ou = O + unit_off(g.os, b, h);
+    const DT *Vu = V + unit_off(g.vs, b, h);
+    const int hi = min(g.T, lo + kFillRows);
+    for (int i = lo + r0; i < hi; i += 32) {
+        DT *dst = Ou + (long long)i * g.os[2];
+        if (i >= L) store8(dst, sub, zero8);
+        else if (chosen[i - lo]) continue;
+        else if (own_v) { float v[8]; load8(Vu + (long long)i * g.vs[2], sub, v); store8(dst, sub, v); }
+        else store8(dst, sub, mean8);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Host-side launchers
+// ---------------------------------------------------------------------------------------
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
+
+template <typename DT>
+static cudaError_t launch_measure_t(const Geom &g, const void *Q, const void *K, const int *sidx,
+                                    float *M, cudaStream_t st) {
+    const long long total = (long long)g.B * g.H * g.T;
+    if (total == 0) return cudaSuccess;
+    const unsigned blocks = (unsigned)((total + 7) / 8);
+    k_measure<DT><<<blocks, 256, 0, st>>>(g, (const DT *)Q, (const DT *)K, sidx, M); note_launch();
+    return cudaGetLastError();
+}
+cudaError_t launch_measure(int dtype, const Geom &g, const void *Q, const void *K, const int *sidx,
+                           float *M, cudaStream_t st) {
+    return dtype == 0 ? launch_measure_t<__nv_bfloat16>(g, Q, K, sidx, M, st)
+                      : launch_measure_t<float>(g, Q, K, sidx, M, st);
+}
+
+cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, int n_chunks,
+                          cudaStream_t st) {
+    if (g.B * g.H == 0 || n_chunks == 0) return cudaSuccess;
+    dim3 grid((unsigned)(g.B * g.H), (unsigned)n_chunks);
+    if (dtype == 0) k_colsum<__nv_bfloat16><<<grid, 256, 0, st>>>(g, (const __nv_bfloat16 *)V, part, n_chunks);
+    else k_colsum<float><<<grid, 256, 0, st>>>(g, (const float *)V, part, n_chunks);
+    note_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,
+                          float *vbar, cudaStream_t st) {
+    if (g.B * g.H == 0) return cudaSuccess;
+    k_select<<<(unsigned)(g.B * g.H), kSelectThreads, 0, st>>>(g, M, sel, vpart, n_chunks, vbar); note_launch();
+    return cudaGetLastError();
+}
+
+template <typename DT, typename OT>
+static cudaError_t launch_attend_t(const Geom &g, const void *Q, const void *K, const void *V,
+                                   const int *rows, int n_rows, int rows_stride, int n_splits,
+                                   int split_keys, float *part_ml, float *part_acc, void *out,
+                                   long long ous, long long ors, int by_pos, cudaStream_t st) {
+    const long long warps = (long long)g.B * g.H * n_rows * n_splits;
+    if (warps == 0) return cudaSuccess;
+    k_attend<DT, OT><<<(unsigned)((warps + 3) / 4), 128, 0, st>>>(
+        g, (const DT *)Q, (const DT *)K, (const DT *)V, rows, n_rows, rows_stride, n_splits,
+        split_keys, part_ml, part_acc, (OT *)out, ous, ors, by_pos); note_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || n_splits == 1) return e;
+    const long long threads = (long long)g.B * g.H * n_rows * kD;
+    k_attend_combine<OT><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
+        g, rows, n_rows, rows_stride, n_splits, part_ml, part_acc, (OT *)out, ous, ors, by_pos); note_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_attend_simt(int dtype, int out_fp32, const Geom &g, const void *Q, const void *K,
+                               const void *V, const int *rows, int n_rows, int rows_stride,
+                               int n_splits, int split_keys, float *part_ml, float *part_acc,
+                               void *out, long long out_unit_stride, long long out_row_stride,
+                               int out_by_position, cudaStream_t st) {
+#define PSATTN_ATT(DT, OT)                                                                      \
+    launch_attend_t<DT, OT>(g, Q, K, V, rows, n_rows, rows_stride, n_splits, split_keys, part_ml, \
+                            part_acc, out, out_unit_stride, out_row_stride, out_by_position, st)
+    if (dtype == 0) return out_fp32 ? PSATTN_ATT(__nv_bfloat16, float) : PSATTN_ATT(__nv_bfloat16, __nv_bfloat16);
+    return PSATTN_ATT(float, float);
+#undef PSATTN_ATT
+}
+
+cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
+                        void *O, int own_v, cudaStream_t st) {
+    if (g.B * g.H == 0 || g.T == 0) return cudaSuccess;
+    dim3 grid((unsigned)(g.B * g.H), (unsigned)((g.T + kFillRows - 1) / kFillRows));
+    if (dtype == 0)
+        k_fill<__nv_bfloat16><<<grid, 256, 0, st>>>(g, (const __nv_bfloat16 *)V, sel, vbar, (__nv_bfloat16 *)O, own_v);
+    else
+        k_fill<float><<<grid, 256, 0, st>>>(g, (const float *)V, sel, vbar, (float *)O, own_v);
+    note_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace psattn

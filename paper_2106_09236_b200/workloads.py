@@ -60,12 +60,13 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
 
 
 def make_inputs(w: Workload, n_cols: int, seed: int | None = None, B: int | None = None,
-                pad_value: float = 0.0):
+                pad_value: float = 0.0, lengths=None):
     """Draw one batch.
 
     n_cols  number of sampled-key columns drawn for every query (the caller
             derives it from the sample-size rule of whichever side it tests).
     B       optional override of the batch size (same per-sequence recipe).
+    lengths optional explicit valid lengths (then none are drawn).
     Returns a dict of numpy arrays: Q, K, V float32 [B,H,T,d] (already rounded
     to bf16 values when w.dtype == "bf16"), lengths int32 [B], sample_idx int32
     [B,T,n_cols] with every entry of row (b, i) in [0, lengths[b]), and `peaky`
@@ -75,7 +76,10 @@ def make_inputs(w: Workload, n_cols: int, seed: int | None = None, B: int | None
     rng = np.random.default_rng(w.seed if seed is None else seed)
     nb = w.B if B is None else B
     H, T, d = w.H, w.T, w.d
-    if w.ragged is not None:
+    if lengths is not None:
+        lengths = np.asarray(lengths, dtype=np.int32)
+        nb = int(lengths.shape[0])
+    elif w.ragged is not None:
         lengths = rng.integers(w.ragged[0], w.ragged[1] + 1, size=nb).astype(np.int32)
     else:
         lengths = np.full(nb, T, dtype=np.int32)

@@ -1,0 +1,365 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+Every test here needs a B200; inputs are seeded and synthetic (paper_2106_09236_b200.workloads).
+"""
+import numpy as np
+import pytest
+import torch
+
+import parity
+from oracle import psattn_oracle as orc
+from paper_2106_09236_b200 import binding as ps
+from paper_2106_09236_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+PATHS = [ps.PSATTN_PATH_STAGED, ps.PSATTN_PATH_AUTO]
+PATH_IDS = ["staged", "auto"]
+
+
+def _dev(inp, dtype):
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    out = {k: torch.from_numpy(inp[k]).to("cuda", tdt) for k in ("Q", "K", "V")}
+    out["lengths"] = torch.from_numpy(inp["lengths"]).cuda()
+    out["sample_idx"] = torch.from_numpy(inp["sample_idx"]).cuda()
+    return out, tdt
+
+
+def _synth(B, H, T, seed, n_cols, dtype="bf16", lengths=None, scale_peaky=3.0):
+    w = wl.Workload("adhoc", 0, B, H, T, 64, dtype, 5.0, 0.1, scale_peaky)
+    return wl.make_inputs(w, n_cols, seed=seed, lengths=lengths)
+
+
+def _run_forward(inp, dtype, c, path, want_M=True, **plan_kw):
+    dev, tdt = _dev(inp, dtype)
+    B, H, T, d = inp["Q"].shape
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=inp["sample_idx"].shape[-1], path=path, **plan_kw)
+    M = torch.full((B, H, T), float("nan"), dtype=torch.float32, device="cuda") if want_M else None
+    O = torch.full((B, H, T, d), float("nan"), dtype=tdt, device="cuda")
+    sel = torch.full((B, H, plan.u_max), -7, dtype=torch.int32, device="cuda")
+    plan.psattn_forward(dev["Q"], dev["K"], dev["V"], dev["lengths"], dev["sample_idx"], O, sel, M)
+    torch.cuda.synchronize()
+    status = plan.psattn_read_status()
+    res = (O.float().cpu().numpy(), sel.cpu().numpy(), None if M is None else M.cpu().numpy(), status)
+    plan.close()
+    return res
+
+
+# ---- the five workloads, full size ---------------------------------------------------------
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("name", ["tiny_fp32", "base_bf16", "ragged_bf16", "large_bf16", "long_bf16"])
+def test_forward_matches_oracle_on_workload(name, path):
+    w = wl.WORKLOADS[name]
+    n_cols = max(orc.count(w.c, L) for L in range(1, w.T + 1))
+    inp = wl.make_inputs(w, n_cols)
+    O, sel, M, status = _run_forward(inp, w.dtype, w.c, path)
+    assert status == 0
+    info = parity.check_forward(O, sel, M, inp, inp["lengths"], w.dtype, w.c)
+    assert info["swapped_units"] <= max(1, (w.B * w.H) // 8)
+
+
+# ---- ragged sizes, several tiles and tails ------------------------------------------------
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("T", [1, 2, 3, 17, 127, 129, 300, 1100, 2500])
+def test_forward_small_and_ragged(T, dtype, path):
+    B, H, c = 3, 2, 5.0
+    lengths = [T, max(1, T // 2), max(1, T - 1)]
+    n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+    inp = _synth(B, H, T, 500 + T, n_cols, dtype, lengths)
+    O, sel, M, status = _run_forward(inp, dtype, c, path)
+    assert status == 0
+    parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_padding_contents_are_never_read(path):
+    B, H, T, c = 2, 2, 200, 5.0
+    lengths = [77, 200]
+    n_cols = orc.count(c, T)
+    inp = _synth(B, H, T, 42, n_cols, "bf16", lengths)
+    ref = _run_forward(inp, "bf16", c, path)
+    poisoned = {k: v.copy() for k, v in inp.items()}
+    for k in ("Q", "K", "V"):
+        poisoned[k][0, :, 77:] = np.nan
+    poisoned["sample_idx"][0, 77:] = 10 ** 6        # rows of padded queries are never read either
+    got = _run_forward(poisoned, "bf16", c, path)
+    assert got[3] == 0
+    np.testing.assert_array_equal(got[0], ref[0])
+    np.testing.assert_array_equal(got[1], ref[1])
+    np.testing.assert_array_equal(got[2], ref[2])
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_all_selected_equals_dense_attention(path):
+    """u = len: every row goes through step (d); the result is Eq. 6."""
+    B, H, T, c = 2, 2, 96, 5.0
+    lengths = [96, 51]
+    inp = _synth(B, H, T, 43, orc.count(c, T), "fp32", lengths)
+    O, sel, M, status = _run_forward(inp, "fp32", c, path, u_override=T)
+    dense = orc.dense(inp["Q"], inp["K"], inp["V"], inp["lengths"])
+    assert np.abs(O - dense).max() <= parity.O_ATOL["fp32"]
+    for b in range(B):
+        assert [int(x) for x in sel[b, 0] if x >= 0] == list(range(lengths[b]))
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_zero_queries_tie_rule_and_exact_zero_measure(path):
+    B, H, T, c = 1, 2, 150, 5.0
+    inp = _synth(B, H, T, 44, orc.count(c, T), "bf16")
+    inp["Q"][:] = 0.0
+    O, sel, M, status = _run_forward(inp, "bf16", c, path)
+    assert np.all(M == 0.0)
+    u = orc.count(c, T)
+    for h in range(H):
+        assert [int(x) for x in sel[0, h] if x >= 0] == list(range(u))
+    vbar = orc.mean_v(inp["V"])
+    assert np.abs(O - vbar[:, :, None, :]).max() <= parity.O_ATOL["bf16"]
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_duplicate_samples_and_constant_rows(path):
+    B, H, T, c = 1, 2, 64, 5.0
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 45, n, "fp32")
+    inp["sample_idx"][0, :, 1] = inp["sample_idx"][0, :, 0]
+    inp["sample_idx"][0, 5, :] = 9
+    O, sel, M, status = _run_forward(inp, "fp32", c, path)
+    assert np.all(M >= 0.0)
+    assert M[0, 0, 5] == 0.0 and M[0, 1, 5] == 0.0
+    parity.check_forward(O, sel, M, inp, inp["lengths"], "fp32", c)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_own_value_fill_and_sample_override(path):
+    """Eq. 12 as printed (v_i for the rest) with the paper's r_sparse = 0.5 and a small sample."""
+    B, H, T, c = 2, 2, 120, 5.0
+    lengths = [120, 64]
+    inp = _synth(B, H, T, 46, 8, "bf16", lengths)
+    O, sel, M, status = _run_forward(inp, "bf16", c, path, u_override=60, U_override=8,
+                                     fill_mode=ps.PSATTN_FILL_OWN_V)
+    parity.check_forward(O, sel, M, inp, inp["lengths"], "bf16", c, u_override=60, U_override=8,
+                         fill="own_v")
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_out_of_range_inputs_set_status_bits_without_faulting(path):
+    B, H, T, c = 2, 1, 80, 5.0
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 47, n, "bf16")
+    bad = {k: v.copy() for k, v in inp.items()}
+    bad["sample_idx"][0, 3, 2] = T + 1000
+    bad["sample_idx"][1, 7, 0] = -5
+    O, sel, M, status = _run_forward(bad, "bf16", c, path)
+    assert status & 1
+    fixed = {k: v.copy() for k, v in inp.items()}
+    fixed["sample_idx"][0, 3, 2] = T - 1             # clamped to the last valid key
+    fixed["sample_idx"][1, 7, 0] = 0                 # clamped to the first key
+    O2, sel2, M2, status2 = _run_forward(fixed, "bf16", c, path)
+    assert status2 == 0
+    np.testing.assert_array_equal(M, M2)
+    np.testing.assert_array_equal(O, O2)
+    too_long = {k: v.copy() for k, v in inp.items()}
+    too_long["lengths"] = np.array([T + 5, -3], dtype=np.int32)
+    O3, sel3, M3, status3 = _run_forward(too_long, "bf16", c, path)
+    assert status3 & 2
+    assert np.all(O3[1] == 0.0) and np.all(sel3[1] == -1)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_run_to_run_determinism(path):
+    w = wl.WORKLOADS["base_bf16"]
+    n = orc.count(w.c, w.T)
+    inp = wl.make_inputs(w, n, B=4)
+    a = _run_forward(inp, "bf16", w.c, path)
+    b = _run_forward(inp, "bf16", w.c, path)
+    for x, y in zip(a[:3], b[:3]):
+        np.testing.assert_array_equal(x, y)
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_strided_bthd_layout(path):
+    """Q, K, V, O stored [B][T][H][d] (projection output order) through the stride fields."""
+    B, H, T, c, d = 2, 4, 160, 5.0, 64
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 48, n, "bf16", [160, 90])
+    dev, tdt = _dev(inp, "bf16")
+    st = (T * H * d, d, H * d)
+    perm = {k: dev[k].permute(0, 2, 1, 3).contiguous() for k in ("Q", "K", "V")}   # [B,T,H,d]
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n, path=path,
+                   strides={"q": st, "k": st, "v": st, "o": st})
+    O = torch.full((B, T, H, d), float("nan"), dtype=tdt, device="cuda")
+    sel = torch.empty((B, H, plan.u_max), dtype=torch.int32, device="cuda")
+    M = torch.empty((B, H, T), dtype=torch.float32, device="cuda")
+    plan.psattn_forward(perm["Q"], perm["K"], perm["V"], dev["lengths"], dev["sample_idx"], O, sel, M)
+    torch.cuda.synchronize()
+    parity.check_forward(O.permute(0, 2, 1, 3).float().cpu().numpy(), sel.cpu().numpy(),
+                         M.cpu().numpy(), inp, inp["lengths"], "bf16", c)
+    plan.close()
+
+
+# ---- per-step entry points -----------------------------------------------------------------------
+
+def test_measure_entry_point():
+    w = wl.WORKLOADS["base_bf16"]
+    n = orc.count(w.c, w.T)
+    inp = wl.make_inputs(w, n, B=3)
+    dev, tdt = _dev(inp, "bf16")
+    plan = ps.Plan(3, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n)
+    M = plan.psattn_measure(dev["Q"], dev["K"], dev["lengths"], dev["sample_idx"])
+    torch.cuda.synchronize()
+    parity.check_measure(M.cpu().numpy(), orc.measure(inp["Q"], inp["K"], inp["sample_idx"],
+                                                      inp["lengths"], c=w.c), inp["lengths"])
+    plan.close()
+
+
+def test_measure_per_head_samples():
+    B, H, T, c = 2, 3, 70, 5.0
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 49, n, "fp32")
+    rng = np.random.default_rng(2)
+    idx = rng.integers(0, T, size=(B, H, T, n)).astype(np.int32)
+    plan = ps.Plan(B, H, T, dtype=torch.float32, c=c, idx_cols=n, idx_per_head=True)
+    M = plan.psattn_measure(torch.from_numpy(inp["Q"]).cuda(), torch.from_numpy(inp["K"]).cuda(),
+                            None, torch.from_numpy(idx).cuda())
+    torch.cuda.synchronize()
+    parity.check_measure(M.cpu().numpy(), orc.measure(inp["Q"], inp["K"], idx, None, c=c))
+    plan.close()
+
+
+def test_select_entry_point_is_exact_including_ties():
+    B, H, T, c = 3, 2, 700, 5.0
+    rng = np.random.default_rng(50)
+    M = rng.standard_normal((B, H, T)).astype(np.float32)
+    M[0, 0] = np.round(M[0, 0] * 2) / 2            # heavy ties
+    M[1, 1] = 0.0                                   # all equal
+    M[2, 0, ::3] = -M[2, 0, ::3] * 1e-30            # tiny values of both signs
+    M[2, 1] = -np.abs(M[2, 1])                      # all negative
+    lengths = np.array([700, 333, 41], dtype=np.int32)
+    plan = ps.Plan(B, H, T, c=c)
+    sel = plan.psattn_select(torch.from_numpy(M).cuda(), torch.from_numpy(lengths).cuda())
+    torch.cuda.synchronize()
+    ref = orc.select(M.astype(np.float64), lengths, c=c, u_max=plan.u_max)
+    np.testing.assert_array_equal(sel.cpu().numpy(), ref)
+    plan.close()
+
+
+def test_mean_v_entry_point():
+    B, H, T = 3, 2, 900
+    inp = _synth(B, H, T, 51, 4, "bf16", [900, 257, 1])
+    dev, tdt = _dev(inp, "bf16")
+    plan = ps.Plan(B, H, T, dtype=tdt, c=5.0)
+    vbar = plan.psattn_mean_v(dev["V"], dev["lengths"])
+    torch.cuda.synchronize()
+    ref = orc.mean_v(inp["V"], inp["lengths"])
+    assert np.abs(vbar.cpu().numpy() - ref).max() <= 1e-5
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_attend_rows_entry_point(dtype):
+    B, H, T, c = 2, 2, 1500, 5.0
+    lengths = [1500, 1029]
+    inp = _synth(B, H, T, 52, 4, dtype, lengths)
+    dev, tdt = _dev(inp, dtype)
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c)
+    rng = np.random.default_rng(3)
+    n_rows = min(9, plan.u_max)
+    rows = np.stack([[rng.choice(lengths[b], size=n_rows, replace=False) for _ in range(H)]
+                     for b in range(B)]).astype(np.int32)
+    rows[1, 0, 2] = -1                               # skipped slot -> zero row
+    rows[1, 1, 4] = 1400                             # beyond the valid length -> zero row
+    out = plan.psattn_attend_rows(dev["Q"], dev["K"], dev["V"], dev["lengths"],
+                                  torch.from_numpy(rows).cuda())
+    torch.cuda.synchronize()
+    out = out.cpu().numpy()
+    tol = 1e-4 if dtype == "fp32" else 2e-3          # fp32 output rows: no bf16 output rounding
+    for b in range(B):
+        for h in range(H):
+            for r in range(n_rows):
+                i = int(rows[b, h, r])
+                if i < 0 or i >= lengths[b]:
+                    assert np.all(out[b, h, r] == 0.0)
+                else:
+                    ref = orc.attend_row(inp["Q"], inp["K"], inp["V"], b, h, i, lengths[b])
+                    assert np.abs(out[b, h, r] - ref).max() <= tol
+    plan.close()
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+def test_forward_with_given_selection(path):
+    """Sec. 4.4: a selection computed once is reused; also covers arbitrary (random) index sets."""
+    B, H, T, c = 2, 2, 260, 5.0
+    lengths = [260, 130]
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 53, n, "bf16", lengths)
+    dev, tdt = _dev(inp, "bf16")
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n, path=path)
+    rng = np.random.default_rng(4)
+    sel_in = np.full((B, H, plan.u_max), -1, dtype=np.int32)
+    for b in range(B):
+        for h in range(H):
+            k = orc.count(c, lengths[b])
+            sel_in[b, h, :k] = np.sort(rng.choice(lengths[b], size=k, replace=False))
+    O = plan.psattn_forward_with_selection(dev["Q"], dev["K"], dev["V"], dev["lengths"],
+                                           torch.from_numpy(sel_in).cuda())
+    torch.cuda.synchronize()
+    O_ref, _, _ = orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"],
+                              c=c, sel_in=sel_in)
+    parity.check_outputs(O.float().cpu().numpy(), O_ref, {}, inp, inp["lengths"], "bf16")
+    plan.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_dense_comparator(dtype):
+    B, H, T = 2, 2, 300
+    lengths = [300, 171]
+    inp = _synth(B, H, T, 54, 4, dtype, lengths)
+    dev, tdt = _dev(inp, dtype)
+    plan = ps.Plan(B, H, T, dtype=tdt, c=5.0)
+    O = plan.psattn_dense_forward(dev["Q"], dev["K"], dev["V"], dev["lengths"])
+    torch.cuda.synchronize()
+    ref = orc.dense(inp["Q"], inp["K"], inp["V"], inp["lengths"])
+    assert np.abs(O.float().cpu().numpy() - ref).max() <= parity.O_ATOL[dtype]
+    plan.close()
+
+
+def test_host_buffer_front_end():
+    w = wl.WORKLOADS["ragged_bf16"]
+    n = max(orc.count(w.c, L) for L in range(1, w.T + 1))
+    inp = wl.make_inputs(w, n, B=4)
+    tdt = torch.bfloat16
+    plan = ps.Plan(4, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n)
+    plan.psattn_plan_enable_host_io()
+    hQ, hK, hV = (torch.from_numpy(inp[k]).to(tdt).pin_memory() for k in ("Q", "K", "V"))
+    hl = torch.from_numpy(inp["lengths"]).pin_memory()
+    hi = torch.from_numpy(inp["sample_idx"]).pin_memory()
+    hO = torch.empty((4, w.H, w.T, 64), dtype=tdt).pin_memory()
+    hs = torch.empty((4, w.H, plan.u_max), dtype=torch.int32).pin_memory()
+    plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs)
+    parity.check_forward(hO.float().numpy(), hs.numpy(), None, inp, inp["lengths"], "bf16", w.c)
+    plan.close()
+
+
+def test_argument_errors_are_status_codes():
+    plan = ps.Plan(1, 1, 64, c=5.0)
+    x = torch.zeros((1, 1, 64, 64), dtype=torch.bfloat16, device="cuda")
+    idx = torch.zeros((1, 64, plan.idx_cols), dtype=torch.int32, device="cuda")
+    with pytest.raises(ps.PsattnError, match="NULL"):
+        plan.psattn_forward(x, x, None, None, idx)
+    with pytest.raises(ps.PsattnError, match="aligned"):
+        plan.psattn_measure(x.view(-1)[1:], x, None, idx)
+    small = plan.workspace
+    plan.workspace_bytes_saved = plan.workspace_bytes
+    plan.workspace_bytes = 16
+    with pytest.raises(ps.PsattnError, match="workspace"):
+        plan.psattn_forward(x, x, x, None, idx)
+    plan.workspace_bytes = plan.workspace_bytes_saved
+    with pytest.raises(ps.PsattnError):
+        ps.Plan(1, 1, 64, d_head=32)
+    with pytest.raises(ps.PsattnError):
+        ps.Plan(1, 1, 64, idx_cols=3)                # narrower than the rule's U
+    del small
+    plan.close()

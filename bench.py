@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the prob-sparse attention forward path (steps (a)-(e) of Sec. 3 of the paper).
+
+One "step" = one psattn_forward over one batch of a seeded synthetic workload.
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+For N > 1 launch with torch.distributed.run; every rank runs the same per-GPU batch (weak
+scaling, no collective on the data path: (batch, head) units are independent).
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2106_09236_b200 import workloads as wl  # noqa: E402
+
+METRIC = "prob-sparse attention queries/s"
+UNIT = "queries/s"
+L2_BYTES = 126e6
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def algorithmic_bytes(w, lengths, count, elem):
+    """Bytes the method itself must move: Q, K, V read once, O written once, the used part of
+    sample_idx (shared by heads), sel_idx, lengths."""
+    total = 0
+    for L in lengths:
+        L = int(L)
+        n = count(w.c, L)
+        total += w.H * L * w.d * (3 * elem + elem) + L * n * 4 + w.H * n * 4
+    return total + 4 * len(lengths)
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                break
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def cpu_oracle_timing(w, n_cols, steps=1, warmup=0):
+    from oracle import psattn_oracle as orc
+    inp = wl.make_inputs(w, n_cols)
+    cores = orc.max_threads()
+    queries = int(inp["lengths"].sum()) * w.H
+    for _ in range(warmup):
+        orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c, nthreads=cores)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c, nthreads=cores)
+    dt = (time.perf_counter() - t0) / steps
+    return queries / dt, cores, dt, queries
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import psattn_oracle as orc
+    n_cols = max(orc.count(w.c, L) for L in range(1, w.T + 1))
+    steps = max(1, min(args.steps, 5))
+    warm = max(0, min(args.warmup, 1))
+    qps, cores, dt, queries = cpu_oracle_timing(w, n_cols, steps, warm)
+    sample = "whole batch of %s (%d valid queries) per step" % (w.name, queries)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "d_head": w.d, "c": w.c},
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def time_events(fn, steps, torch):
+    """Runs fn(k) for k in range(steps) between two CUDA events on the current stream."""
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record()
+    for k in range(steps):
+        fn(k)
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end) / steps      # ms per step
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large_bf16", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
+    ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of CUDA-graph replays")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense comparator timing")
+    args = ap.parse_args()
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2106_09236_b200 import binding as ps
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    elem = 2 if w.dtype == "bf16" else 4
+    n_cols = max(ps.psattn_count(w.c, L) for L in range(1, w.T + 1))
+    path = {"auto": ps.PSATTN_PATH_AUTO, "staged": ps.PSATTN_PATH_STAGED, "fused": ps.PSATTN_PATH_FUSED}[args.path]
+    plan = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, path=path)
+
+    # enough independent buffer sets that a set is evicted from L2 before it is used again
+    per_set = 4 * w.B * w.H * w.T * w.d * elem + w.B * w.T * n_cols * 4
+    n_sets = max(2, int(np.ceil(2.2 * L2_BYTES / per_set)) + 1)
+    sets, host_sets, queries_per_step, alg_bytes = [], [], None, None
+    for s in range(n_sets):
+        inp = wl.make_inputs(w, n_cols, seed=w.seed + 1000 * rank + 17 * s)
+        if s == 0:
+            host_sets.append(inp)
+            queries_per_step = int(inp["lengths"].sum()) * w.H
+            alg_bytes = algorithmic_bytes(w, inp["lengths"], ps.psattn_count, elem)
+        d = {k: torch.from_numpy(inp[k]).to("cuda", tdt) for k in ("Q", "K", "V")}
+        d["lengths"] = torch.from_numpy(inp["lengths"]).cuda()
+        d["sample_idx"] = torch.from_numpy(inp["sample_idx"]).cuda()
+        d["O"] = torch.empty((w.B, w.H, w.T, w.d), dtype=tdt, device="cuda")
+        d["sel"] = torch.empty((w.B, w.H, plan.u_max), dtype=torch.int32, device="cuda")
+        sets.append(d)
+
+    def step(k):
+        d = sets[k % n_sets]
+        plan.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], d["sel"])
+
+    l0 = ps.psattn_launch_count()
+    step(0)
+    torch.cuda.synchronize()
+    launches_per_step = ps.psattn_launch_count() - l0
+
+    graphs = None
+    if not args.no_graph:
+        graphs = []
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for s in range(n_sets):
+                step(s)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        for s in range(n_sets):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                step(s)
+            graphs.append(g)
+
+    def timed_step(k):
+        if graphs is not None:
+            graphs[k % n_sets].replay()
+        else:
+            step(k)
+
+    for k in range(max(args.warmup, 3)):
+        timed_step(k)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms = time_events(timed_step, args.steps, torch)
+    clocks = sampler.stop()
+    if world > 1:
+        dist.barrier()
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    status = plan.psattn_read_status()
+    value = queries_per_step * world / (ms * 1e-3)
+
+    # direct (non-graph) C-ABI calls, for the record
+    direct_ms = time_events(step, min(args.steps, 200), torch)
+
+    # per-entry-point times (same kernels), rotating buffers, to find the dominant kernel
+    M_buf = torch.empty((w.B, w.H, w.T), dtype=torch.float32, device="cuda")
+
+    def k_measure(k):
+        d = sets[k % n_sets]
+        plan.psattn_measure(d["Q"], d["K"], d["lengths"], d["sample_idx"], M_buf)
+
+    def k_rest(k):
+        d = sets[k % n_sets]
+        plan.psattn_forward_with_selection(d["Q"], d["K"], d["V"], d["lengths"], d["sel"], d["O"])
+
+    nk = min(args.steps, 200)
+    for k in range(3):
+        k_measure(k); k_rest(k)
+    kernel_ms = {"measure(a+b)": time_events(k_measure, nk, torch),
+                 "mean_v+attend+fill(d+e)": time_events(k_rest, nk, torch)}
+    peak, peak_kind = measured_peaks()
+    units = w.B * w.H
+    measure_bytes = units * w.T * w.d * elem * 2 + w.B * w.T * n_cols * 4 + units * w.T * 4
+    if launches_per_step == 1:
+        roof_kernel, roof_bytes, roof_ms = "fused forward", alg_bytes, ms
+    else:
+        roof_kernel, roof_bytes, roof_ms = "measure (steps a+b)", measure_bytes, kernel_ms["measure(a+b)"]
+    achieved = roof_bytes / (roof_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_kind": "of " + peak_kind,
+                "algorithmic_bytes_per_launch": roof_bytes}
+    path_gbs = alg_bytes / (ms * 1e-3) / 1e9
+
+    # end to end through the host-buffer entry point (pinned host memory, copies timed)
+    e2e = None
+    if True:
+        plan.psattn_plan_enable_host_io()
+        inp = host_sets[0]
+        hQ, hK, hV = (torch.from_numpy(inp[k]).to(tdt).pin_memory() for k in ("Q", "K", "V"))
+        hl = torch.from_numpy(inp["lengths"]).pin_memory()
+        hi = torch.from_numpy(inp["sample_idx"]).pin_memory()
+        hO = torch.empty((w.B, w.H, w.T, w.d), dtype=tdt).pin_memory()
+        hs = torch.empty((w.B, w.H, plan.u_max), dtype=torch.int32).pin_memory()
+        ne = max(3, min(args.steps, 20))
+        for _ in range(3):
+            plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs)
+        if world > 1:
+            dist.barrier()
+        e_ms = time_events(lambda k: plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs), ne, torch)
+        if world > 1:
+            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hl, hi))
+        d2h = sum(x.numel() * x.element_size() for x in (hO, hs))
+        e2e = {"value": queries_per_step * world / (e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": ne}
+
+    dense = None
+    if not args.no_dense and rank == 0:
+        d = sets[0]
+        plan.psattn_dense_forward(d["Q"], d["K"], d["V"], d["lengths"], d["O"])
+        nd = 3
+        d_ms = time_events(lambda k: plan.psattn_dense_forward(
+            sets[k % n_sets]["Q"], sets[k % n_sets]["K"], sets[k % n_sets]["V"],
+            sets[k % n_sets]["lengths"], sets[k % n_sets]["O"]), nd, torch)
+        dense = {"ms_per_step": d_ms, "speedup_sparse_vs_dense": d_ms / ms,
+                 "workspace_bytes_sparse": plan.workspace_bytes}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        qps, cores, dt, q = cpu_oracle_timing(w, n_cols)
+        cpu = {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "whole batch of %s (%d valid queries), one pass, %.2f s" % (w.name, q, dt)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "d_head": w.d, "c": w.c,
+                       "U": n_cols, "path": args.path, "graph_replay": graphs is not None,
+                       "l2": "rotating %d independent buffer sets (%.0f MB > 126 MB L2)" % (
+                           n_sets, n_sets * per_set / 1e6)},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_per_step * args.steps),
+            "roofline": roofline, "cpu_baseline": cpu,
+            "path_effective_gbs": path_gbs, "path_frac_of_hbm": path_gbs / peak,
+            "algorithmic_bytes_per_step": alg_bytes, "queries_per_step": queries_per_step,
+            "kernel_ms": kernel_ms, "direct_call_ms_per_step": direct_ms, "dense": dense,
+            "device_status": status,
+        }
+        print(json.dumps(line), flush=True)
+    plan.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -59,7 +59,8 @@ enum {
     PSATTN_ERR_WORKSPACE_TOO_SMALL = 4,
     PSATTN_ERR_MISALIGNED = 5,          /* a base pointer is not 16-byte aligned */
     PSATTN_ERR_CUDA = 6,                /* a CUDA runtime call failed; see psattn_last_cuda_error */
-    PSATTN_ERR_NO_DEVICE = 7            /* no usable sm_100 device */
+    PSATTN_ERR_NO_DEVICE = 7,           /* no usable sm_100 device */
+    PSATTN_ERR_TOO_LARGE = 8            /* problem exceeds a fixed built-in capacity */
 };
 
 enum { PSATTN_BF16 = 0, PSATTN_FP32 = 1 };
@@ -166,6 +167,32 @@ int psattn_plan_enable_host_io(psattn_plan_t *plan);
 int psattn_forward_host(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
                         const int32_t *lengths, const int32_t *sample_idx, void *O,
                         int32_t *sel_idx, void *stream);
+
+/* Allocation-free variant of psattn_mean_v.  (The paper has no counterpart: this entry point
+ * exists for deployment reasons only; it computes the same fill value of step (e).)
+ *
+ * For callers that cannot allocate device memory where they need the result - code running
+ * under a framework that owns all device memory through its own pool, pipelines that forbid
+ * allocation after start-up, plug-ins in a process whose memory is already reserved.  It needs
+ * no plan and no workspace: its scratch (the column-sum partials) is a fixed array inside the
+ * library image, PSATTN_NOALLOC_MAX_PARTIALS * 64 floats (4 MiB) plus 256 bytes, which every
+ * GPU that loads the library holds until the process exits.  It calls no cudaMalloc, cudaFree
+ * or other allocating routine.
+ *
+ *   V        device, dense [B][H][T_max][64] of `dtype` (PSATTN_BF16 | PSATTN_FP32), 16-byte aligned
+ *   lengths  device int32 [B] or NULL (all T_max); values are clamped to [0, T_max]
+ *   vbar     device fp32 [B][H][64]: mean of V over the valid rows (zeros where length is 0)
+ *
+ * Capacity: B * H * ceil(T_max / 256) <= PSATTN_NOALLOC_MAX_PARTIALS, otherwise
+ * PSATTN_ERR_TOO_LARGE is returned and nothing is launched.
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the one array:
+ * it keeps the previous call's contents (each call rewrites what it reads and clears its status
+ * word), and two calls whose kernels may overlap on the GPU (different streams without an
+ * ordering between them) race on it - order them. */
+#define PSATTN_NOALLOC_MAX_PARTIALS 16384
+int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, float *vbar, int32_t B,
+                          int32_t H, int32_t T_max, int32_t dtype, void *stream);
 
 #ifdef __cplusplus
 }

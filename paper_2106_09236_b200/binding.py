@@ -21,7 +21,7 @@ EXPORTS = [
     "psattn_plan_create", "psattn_plan_destroy", "psattn_plan_limits", "psattn_workspace_bytes",
     "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_select",
     "psattn_mean_v", "psattn_attend_rows", "psattn_dense_forward", "psattn_read_status",
-    "psattn_plan_enable_host_io", "psattn_forward_host",
+    "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc",
 ]
 
 
@@ -80,6 +80,7 @@ def load(build_if_missing: bool = True):
     lib.psattn_read_status.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.psattn_plan_enable_host_io.argtypes = [vp]
     lib.psattn_forward_host.argtypes = [vp] * 9
+    lib.psattn_mean_v_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
     _lib = lib
     return lib
 
@@ -113,6 +114,16 @@ def psattn_launch_count() -> int:
 
 def psattn_count(c: float, length: int) -> int:
     return load().psattn_count(float(c), int(length))
+
+
+def psattn_mean_v_noalloc(V, lengths, vbar, B, H, T_max):
+    """mean(V) over valid rows without any allocation: no plan, no workspace.  `vbar` (fp32
+    [B, H, 64], device) must be provided by the caller and is filled in place.  For callers
+    that may not allocate device memory; see include/psattn.h for capacity and sharing rules."""
+    dtype = PSATTN_BF16 if V.dtype == torch.bfloat16 else PSATTN_FP32
+    _check(load().psattn_mean_v_noalloc(_ptr(V), _ptr(lengths), _ptr(vbar), int(B), int(H),
+                                        int(T_max), dtype, _stream()))
+    return vbar
 
 
 class Plan:

@@ -41,6 +41,7 @@ extern "C" const char *psattn_status_string(int s) {
         case PSATTN_ERR_MISALIGNED: return "pointer not 16-byte aligned (workspace: 256-byte)";
         case PSATTN_ERR_CUDA: return "CUDA runtime error";
         case PSATTN_ERR_NO_DEVICE: return "no usable CUDA device";
+        case PSATTN_ERR_TOO_LARGE: return "problem exceeds a fixed built-in capacity";
         default: return "unknown status";
     }
 }

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsattn.so")
-SOURCES = ["psattn_api.cu", "psattn_staged.cu", "psattn_noalloc.cu"]
+SOURCES = ["psattn_api.cu", "psattn_staged.cu", "psattn_noalloc.cu", "psattn_attend_tc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",
@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         subprocess.check_call(cmd)
         objs.append(obj)
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart", "-lcuda"])
+    subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart"])
     os.replace(tmp, LIB)
     return LIB
 

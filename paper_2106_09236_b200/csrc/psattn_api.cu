@@ -129,7 +129,12 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     p->u_max = u_max;
     p->U_max = U_max;
     p->n_chunks = (d.T_max + kColsumRows - 1) / kColsumRows;
-    p->n_splits = (d.T_max + kSplitKeys - 1) / kSplitKeys;
+    p->n_splits = (d.T_max + kSplitKeys - 1) / kSplitKeys;       // what the partial buffers are sized for
+    {
+        const int tiles = (d.T_max + 127) / 128;
+        const int tc_splits = tiles < 8 ? tiles : 8;
+        if (tc_splits > p->n_splits) p->n_splits = tc_splits;
+    }
     cudaError_t e = cudaMalloc((void **)&p->d_tables, tab.size() * sizeof(int));
     if (e != cudaSuccess) { delete p; return PSATTN_ERR_CUDA; }
     e = cudaMemcpy(p->d_tables, tab.data(), tab.size() * sizeof(int), cudaMemcpyHostToDevice);
@@ -209,16 +214,46 @@ static T *ws_at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast
         if (e__ != cudaSuccess) return cuda_fail(plan, e__);    \
     } while (0)
 
+// Step (d) for a row list: tensor-core kernel for bf16 inputs (unless the plan asks for the
+// staged SIMT schedule or the layout has no tensor map), SIMT kernel otherwise.
+static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K, const void *V,
+                      const int *rows, int n_rows, int rows_stride, void *out, long long ous,
+                      long long ors, int by_pos, int out_fp32, void *ws, cudaStream_t st) {
+    const psattn_desc_t &d = plan->desc;
+    float *ml = ws_at<float>(ws, plan->off_ml), *acc = ws_at<float>(ws, plan->off_acc);
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
+        // key splits: enough CTAs to cover the SMs about twice, never more splits than 128-key tiles
+        const int tiles = (d.T_max + 127) / 128;
+        const long long ctas = (long long)d.B * d.H * ((n_rows + 127) / 128);
+        int splits = (int)((2 * 148 + ctas - 1) / (ctas > 0 ? ctas : 1));
+        if (splits > plan->n_splits) splits = plan->n_splits;
+        if (splits > tiles) splits = tiles;
+        if (splits < 1 || rows == nullptr) splits = 1;
+        const int split_keys = ((tiles + splits - 1) / splits) * 128;
+        splits = (d.T_max + split_keys - 1) / split_keys;
+        cudaError_t e = launch_attend_tc(g, Q, K, V, rows, n_rows, rows_stride, splits, split_keys, ml, acc, out,
+                                         ous, ors, by_pos, out_fp32, st);
+        if (e == cudaSuccess) {
+            if (splits > 1)
+                PSATTN_CU(merge_attend_splits(!out_fp32, g, rows, n_rows, rows_stride, splits, ml, acc, out, ous,
+                                              ors, by_pos, st));
+            return PSATTN_OK;
+        }
+        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+    }
+    const int splits = rows ? (d.T_max + kSplitKeys - 1) / kSplitKeys : 1;
+    PSATTN_CU(launch_attend_simt(d.dtype, out_fp32, g, Q, K, V, rows, n_rows, rows_stride, splits,
+                                 rows ? kSplitKeys : d.T_max, ml, acc, out, ous, ors, by_pos, st));
+    return PSATTN_OK;
+}
+
 // Steps (d)+(e) for a selection that already sits in `sel` (device) with vbar in the workspace.
 static int run_attend_and_fill(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K,
                                const void *V, const int *sel, void *O, void *ws, cudaStream_t st) {
     const psattn_desc_t &d = plan->desc;
     PSATTN_CU(launch_fill(d.dtype, g, V, sel, ws_at<float>(ws, plan->off_vbar), O,
                           d.fill_mode == PSATTN_FILL_OWN_V, st));
-    PSATTN_CU(launch_attend_simt(d.dtype, 0, g, Q, K, V, sel, plan->u_max, plan->u_max,
-                                 plan->n_splits, kSplitKeys, ws_at<float>(ws, plan->off_ml),
-                                 ws_at<float>(ws, plan->off_acc), O, 0, 0, 1, st));
-    return PSATTN_OK;
+    return run_attend(plan, g, Q, K, V, sel, plan->u_max, plan->u_max, O, 0, 0, 1, 0, ws, st);
 }
 
 extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
@@ -306,11 +341,8 @@ extern "C" int psattn_attend_rows(psattn_plan_t *plan, const void *Q, const void
     if (rc) return rc;
     if (n_rows == 0) return PSATTN_OK;
     Geom g = make_geom(plan, lengths, workspace);
-    PSATTN_CU(launch_attend_simt(plan->desc.dtype, 1, g, Q, K, V, row_idx, n_rows, n_rows,
-                                 plan->n_splits, kSplitKeys, ws_at<float>(workspace, plan->off_ml),
-                                 ws_at<float>(workspace, plan->off_acc), out,
-                                 (long long)n_rows * kD, kD, 0, static_cast<cudaStream_t>(stream)));
-    return PSATTN_OK;
+    return run_attend(plan, g, Q, K, V, row_idx, n_rows, n_rows, out, (long long)n_rows * kD, kD, 0, 1,
+                      workspace, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const void *K,
@@ -330,9 +362,7 @@ extern "C" int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const vo
     PSATTN_CU(cudaMemsetAsync(sel, 0xff, (size_t)d.B * d.H * plan->u_max * sizeof(int), st));
     PSATTN_CU(cudaMemsetAsync(ws_at<float>(workspace, plan->off_vbar), 0, (size_t)d.B * d.H * kD * sizeof(float), st));
     PSATTN_CU(launch_fill(d.dtype, g, V, sel, ws_at<float>(workspace, plan->off_vbar), O, 0, st));
-    PSATTN_CU(launch_attend_simt(d.dtype, 0, g, Q, K, V, nullptr, d.T_max, 0, 1, d.T_max, nullptr,
-                                 nullptr, O, 0, 0, 1, st));
-    return PSATTN_OK;
+    return run_attend(plan, g, Q, K, V, nullptr, d.T_max, 0, O, 0, 0, 1, 0, workspace, st);
 }
 
 extern "C" int psattn_read_status(psattn_plan_t *plan, void *workspace, void *stream,

@@ -27,6 +27,18 @@ cudaError_t launch_attend_simt(int dtype, int out_fp32, const Geom &g, const voi
                                int n_splits, int split_keys, float *part_ml, float *part_acc,
                                void *out, long long out_unit_stride, long long out_row_stride,
                                int out_by_position, cudaStream_t st);
+// Tensor-core (tcgen05) form of the same step for bf16 inputs; same argument meaning, plus
+// out_fp32 for row-list output.  split_keys must be a multiple of 128.  Returns
+// cudaErrorNotSupported when the layout cannot be described by a TMA tensor map (the caller then
+// uses launch_attend_simt); the split partials are merged by merge_attend_splits.
+cudaError_t launch_attend_tc(const Geom &g, const void *Q, const void *K, const void *V, const int *rows,
+                             int n_rows, int rows_stride, int n_splits, int split_keys, float *part_ml,
+                             float *part_acc, void *out, long long out_unit_stride, long long out_row_stride,
+                             int out_by_position, int out_fp32, cudaStream_t st);
+cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows, int n_rows, int rows_stride,
+                                int n_splits, const float *part_ml, const float *part_acc, void *out,
+                                long long out_unit_stride, long long out_row_stride, int out_by_position,
+                                cudaStream_t st);
 cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
                         void *O, int own_v, cudaStream_t st);
 

@@ -446,6 +446,25 @@ cudaError_t launch_attend_simt(int dtype, int out_fp32, const Geom &g, const voi
 #undef PSATTN_ATT
 }
 
+cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows, int n_rows, int rows_stride,
+                                int n_splits, const float *part_ml, const float *part_acc, void *out,
+                                long long out_unit_stride, long long out_row_stride, int out_by_position,
+                                cudaStream_t st) {
+    const long long threads = (long long)g.B * g.H * n_rows * kD;
+    if (threads == 0) return cudaSuccess;
+    const unsigned blocks = (unsigned)((threads + 255) / 256);
+    if (out_is_bf16)
+        k_attend_combine<__nv_bfloat16><<<blocks, 256, 0, st>>>(g, rows, n_rows, rows_stride, n_splits, part_ml,
+                                                                 part_acc, (__nv_bfloat16 *)out, out_unit_stride,
+                                                                 out_row_stride, out_by_position);
+    else
+        k_attend_combine<float><<<blocks, 256, 0, st>>>(g, rows, n_rows, rows_stride, n_splits, part_ml, part_acc,
+                                                        (float *)out, out_unit_stride, out_row_stride,
+                                                        out_by_position);
+    note_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
                         void *O, int own_v, cudaStream_t st) {
     if (g.B * g.H == 0 || g.T == 0) return cudaSuccess;

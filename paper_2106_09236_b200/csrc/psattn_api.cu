@@ -214,6 +214,19 @@ static T *ws_at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast
         if (e__ != cudaSuccess) return cuda_fail(plan, e__);    \
     } while (0)
 
+// Steps (a)+(b): resident-key kernel for bf16 inputs when it applies, gather-from-L2 kernel otherwise.
+static int run_measure(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K,
+                       const int *sample_idx, float *M, cudaStream_t st) {
+    const psattn_desc_t &d = plan->desc;
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
+        cudaError_t e = launch_measure_mma(g, plan->U_max, Q, K, sample_idx, M, st);
+        if (e == cudaSuccess) return PSATTN_OK;
+        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+    }
+    PSATTN_CU(launch_measure(d.dtype, g, Q, K, sample_idx, M, st));
+    return PSATTN_OK;
+}
+
 // Step (d) for a row list: tensor-core kernel for bf16 inputs (unless the plan asks for the
 // staged SIMT schedule or the layout has no tensor map), SIMT kernel otherwise.
 static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K, const void *V,
@@ -268,7 +281,7 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
     float *M = M_out ? M_out : ws_at<float>(workspace, plan->off_M);
-    PSATTN_CU(launch_measure(d.dtype, g, Q, K, sample_idx, M, st));
+    if ((rc = run_measure(plan, g, Q, K, sample_idx, M, st)) != PSATTN_OK) return rc;
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
     PSATTN_CU(launch_select(g, M, sel_idx, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks,
                             ws_at<float>(workspace, plan->off_vbar), st));
@@ -302,8 +315,7 @@ extern "C" int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K,
     int rc = check_ws(plan, workspace, workspace_bytes);
     if (rc) return rc;
     Geom g = make_geom(plan, lengths, workspace);
-    PSATTN_CU(launch_measure(plan->desc.dtype, g, Q, K, sample_idx, M_out, static_cast<cudaStream_t>(stream)));
-    return PSATTN_OK;
+    return run_measure(plan, g, Q, K, sample_idx, M_out, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,

@@ -15,6 +15,11 @@ unsigned long long launches_so_far();
 
 cudaError_t launch_measure(int dtype, const Geom &g, const void *Q, const void *K, const int *sidx,
                            float *M, cudaStream_t st);
+// Resident-key tensor-datapath form of steps (a)+(b) for bf16 inputs; cudaErrorNotSupported when
+// T_max is too long for shared memory, U_max > 64 or the layout has no tensor map (the caller then
+// uses launch_measure).
+cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
+                               cudaStream_t st);
 cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, int n_chunks,
                           cudaStream_t st);
 cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,

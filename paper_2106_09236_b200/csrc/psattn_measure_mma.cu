@@ -19,11 +19,11 @@ namespace psattn {
 
 using namespace sm100;
 
-constexpr int kMeasureThreads = 1024;
+constexpr int kMeasureThreads = 768;
 constexpr int kMeasureWarps = kMeasureThreads / 32;
 constexpr int kMeasureBoxRows = 256;
 constexpr int kMeasureMaxU = 64;          // four rounds of 16 sampled keys
-constexpr int kMeasureBlock = 64;         // queries staged per step (Q rows + sample rows)
+constexpr int kMeasureBlock = 96;         // queries staged per step (Q rows + sample rows)
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
     // not volatile: what it reads is constant between the barriers around it, and leaving the
@@ -98,29 +98,45 @@ __device__ __forceinline__ void measure_block(const MeasureCtx &cx) {
     const bool last_lo = (ROUNDS - 1) * 16 + dg < cx.U, last_hi = (ROUNDS - 1) * 16 + dg + 8 < cx.U;
     const float inv_U = 1.f / (float)cx.U;
 
-    for (int ql = warp; ql < cx.rows; ql += kMeasureWarps) {
+    // A warp takes kPerWarp consecutive queries of the block.  Their cross-lane reductions are done
+    // together: only one lane per quad (the "diagonal" lane) holds wanted scores, so lane q of each
+    // quad adopts query q's partials from its quad's diagonal lane, and three xor steps across the
+    // quads finish all kPerWarp queries at once.
+    constexpr int kPerWarp = kMeasureBlock / kMeasureWarps;
+    static_assert(kPerWarp == 4, "one query per quad lane");
+    const int quad_src = (lane & ~3) | (dg >> 1);
+    float my_mx = -INFINITY, my_ds = 0.f;
+#pragma unroll
+    for (int k = 0; k < kPerWarp; ++k) {
+        const int ql = min(warp * kPerWarp + k, cx.rows - 1);      // tail: recompute the last row
         uint32_t bq[8];
         ldmatrix_x4(cx.q_tile + (uint32_t)ql * 128u + q_off0, bq[0], bq[1], bq[2], bq[3]);
         ldmatrix_x4(cx.q_tile + (uint32_t)ql * 128u + q_off4, bq[4], bq[5], bq[6], bq[7]);
         const uint32_t krow = cx.idx_tile + (uint32_t)(ql * cx.idx_cols) * 4u;
-        uint32_t row_addr[ROUNDS];
-        float c[ROUNDS][4];
+        int key[ROUNDS];
+        bool bad = false;
 #pragma unroll
         for (int r = 0; r < ROUNDS; ++r) {
-            c[r][0] = c[r][1] = c[r][2] = c[r][3] = 0.f;
-            int key;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(key) : "r"(krow + j_off[r]));
-            if ((unsigned)key >= (unsigned)cx.L) { atomicOr(cx.status, kStatusIdxClamped); key = key < 0 ? 0 : cx.L - 1; }
-            row_addr[r] = cx.k_base + (uint32_t)key * 128u;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(key[r]) : "r"(krow + j_off[r]));
+            bad |= (unsigned)key[r] >= (unsigned)cx.L;
         }
+        if (bad) {                                                 // rare: clamp and report
+            atomicOr(cx.status, kStatusIdxClamped);
+#pragma unroll
+            for (int r = 0; r < ROUNDS; ++r) key[r] = key[r] < 0 ? 0 : min(key[r], cx.L - 1);
+        }
+        float c[ROUNDS][4];
+#pragma unroll
+        for (int r = 0; r < ROUNDS; ++r) c[r][0] = c[r][1] = c[r][2] = c[r][3] = 0.f;
         // the rounds are independent accumulation chains: step t of every round, then step t + 1
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
 #pragma unroll
             for (int r = 0; r < ROUNDS; ++r) {
+                const uint32_t row_addr = cx.k_base + (uint32_t)key[r] * 128u;
                 uint32_t a0, a1 = 0u, a2, a3 = 0u;
-                if (HALF && r == ROUNDS - 1) ldmatrix_x2(row_addr[r] + off_half[t], a0, a2);
-                else ldmatrix_x4(row_addr[r] + off_full[t], a0, a1, a2, a3);
+                if (HALF && r == ROUNDS - 1) ldmatrix_x2(row_addr + off_half[t], a0, a2);
+                else ldmatrix_x4(row_addr + off_full[t], a0, a1, a2, a3);
                 mma_bf16_16816(c[r], a0, a1, a2, a3, bq[2 * t], bq[2 * t + 1]);
             }
         }
@@ -135,18 +151,21 @@ __device__ __forceinline__ void measure_block(const MeasureCtx &cx) {
                 mx = fmaxf(mx, fmaxf(d_lo, d_hi));
                 ds += d_lo + d_hi;
             } else {
-                if (last_lo) { mx = fmaxf(mx, d_lo); ds += d_lo; }
-                if (last_hi) { mx = fmaxf(mx, d_hi); ds += d_hi; }
+                mx = fmaxf(mx, fmaxf(last_lo ? d_lo : -INFINITY, last_hi ? d_hi : -INFINITY));
+                ds += (last_lo ? d_lo : 0.f) + (last_hi ? d_hi : 0.f);
             }
         }
-        if (!diag) { mx = -INFINITY; ds = 0.f; }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            ds += __shfl_xor_sync(0xffffffffu, ds, o);
-        }
-        if (lane == 0) cx.out[ql] = fmaxf((mx - ds * inv_U) * kScale, 0.f);
+        const float q_mx = __shfl_sync(0xffffffffu, mx, quad_src);
+        const float q_ds = __shfl_sync(0xffffffffu, ds, quad_src);
+        if ((lane & 3) == k) { my_mx = q_mx; my_ds = q_ds; }
     }
+#pragma unroll
+    for (int o = 4; o <= 16; o <<= 1) {
+        my_mx = fmaxf(my_mx, __shfl_xor_sync(0xffffffffu, my_mx, o));
+        my_ds += __shfl_xor_sync(0xffffffffu, my_ds, o);
+    }
+    const int ql_out = warp * kPerWarp + lane;
+    if (lane < kPerWarp && ql_out < cx.rows) cx.out[ql_out] = fmaxf((my_mx - my_ds * inv_U) * kScale, 0.f);
 }
 
 __global__ void __launch_bounds__(kMeasureThreads, 1) k_measure_mma(Geom g, MeasureMmaArgs a,

@@ -4,6 +4,7 @@
 //   colsum   : partial column sums of V        fill   : step (e), Eq. 12 else-branch
 //   attend   : step (d), Eq. 7-8, flash-decoding form with one key per lane
 #include "psattn_launch.h"
+#include "psattn_select.cuh"
 
 #include <atomic>
 
@@ -109,36 +110,11 @@ __global__ void __launch_bounds__(256) k_colsum(Geom g, const DT *__restrict__ V
 // (in position order) positions with key == tau, written in ascending position order.
 // The same block finishes mean(V) from the column-sum partials.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ int block_exclusive_scan(int v, int *warp_tot, int &total) {
-    // blockDim.x == kSelectThreads (a multiple of 32, <= 1024); v in {0,1,...}
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    int x = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        int y = __shfl_up_sync(0xffffffffu, x, o);
-        if (lane >= o) x += y;
-    }
-    if (lane == 31) warp_tot[wid] = x;
-    __syncthreads();
-    int before = 0, tot = 0;
-    for (int k = 0; k < nw; ++k) {
-        int t = warp_tot[k];
-        if (k < wid) before += t;
-        tot += t;
-    }
-    __syncthreads();
-    total = tot;
-    return before + x - v;
-}
-
 __global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *__restrict__ M,
                                                            int *__restrict__ sel,
                                                            const float *__restrict__ vpart,
                                                            int n_chunks, float *__restrict__ vbar) {
-    __shared__ int hist[256];
-    __shared__ int warp_tot[32];
-    __shared__ unsigned s_prefix;
-    __shared__ int s_remaining;
+    __shared__ SelectScratch scratch;
     const int unit = blockIdx.x;
     const int b = unit / g.H;
     const int L = seq_len(g, b);
@@ -152,51 +128,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *
         vbar[(long long)unit * kD + threadIdx.x] = L > 0 ? s / (float)L : 0.f;
     }
     if (M == nullptr) return;                  // mean(V) only
-    if (u <= 0) {
-        for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) out[r] = -1;
-        return;
-    }
-    if (threadIdx.x == 0) { s_prefix = 0u; s_remaining = u; }
-    unsigned known = 0u;                       // mask of the key bits fixed so far
-    for (int shift = 24; shift >= 0; shift -= 8) {
-        for (int t = threadIdx.x; t < 256; t += blockDim.x) hist[t] = 0;
-        __syncthreads();
-        const unsigned prefix = s_prefix;
-        for (int i = threadIdx.x; i < L; i += blockDim.x) {
-            unsigned k = float_key(Mu[i]);
-            if (((k ^ prefix) & known) == 0u) atomicAdd(&hist[(k >> shift) & 255u], 1);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            int rem = s_remaining, bin = 255;
-            for (; bin > 0; --bin) {
-                if (hist[bin] >= rem) break;
-                rem -= hist[bin];
-            }
-            s_prefix = prefix | ((unsigned)bin << shift);
-            s_remaining = rem;
-        }
-        known |= 0xffu << shift;
-        __syncthreads();
-    }
-    const unsigned tau = s_prefix;
-    const int need_eq = s_remaining;           // how many of the positions with key == tau to take
-    int eq_seen = 0, written = 0;
-    for (int base = 0; base < L; base += blockDim.x) {
-        const int i = base + threadIdx.x;
-        unsigned k = 0u;
-        const bool valid = i < L;
-        if (valid) k = float_key(Mu[i]);
-        const int is_eq = valid && k == tau;
-        int tot_eq, tot_take;
-        const int eq_rank = eq_seen + block_exclusive_scan(is_eq, warp_tot, tot_eq);
-        const int take = valid && (k > tau || (is_eq && eq_rank < need_eq));
-        const int pos = written + block_exclusive_scan(take, warp_tot, tot_take);
-        if (take && pos < g.u_max) out[pos] = i;
-        eq_seen += tot_eq;
-        written += tot_take;
-    }
-    for (int r = written + threadIdx.x; r < g.u_max; r += blockDim.x) out[r] = -1;
+    block_select([&](int i) { return float_key(Mu[i]); }, L, u, g.u_max, out, scratch);
 }
 
 // ---------------------------------------------------------------------------------------

@@ -234,6 +234,25 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
                       long long ors, int by_pos, int out_fp32, void *ws, cudaStream_t st) {
     const psattn_desc_t &d = plan->desc;
     float *ml = ws_at<float>(ws, plan->off_ml), *acc = ws_at<float>(ws, plan->off_acc);
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && rows != nullptr && n_rows <= 64) {
+        // one CTA per SM: split the keys only when there are fewer units than SMs
+        const int pairs = (d.T_max + 255) / 256;
+        int splits = 148 / (d.B * d.H > 0 ? d.B * d.H : 1);
+        if (splits > plan->n_splits) splits = plan->n_splits;
+        if (splits > pairs) splits = pairs;
+        if (splits < 1) splits = 1;
+        const int split_keys = ((pairs + splits - 1) / splits) * 256;
+        splits = (d.T_max + split_keys - 1) / split_keys;
+        cudaError_t e = launch_attend64(g, Q, K, V, rows, n_rows, rows_stride, splits, split_keys, ml, acc, out, ous,
+                                        ors, by_pos, out_fp32, st);
+        if (e == cudaSuccess) {
+            if (splits > 1)
+                PSATTN_CU(merge_attend_splits(!out_fp32, g, rows, n_rows, rows_stride, splits, ml, acc, out, ous,
+                                              ors, by_pos, st));
+            return PSATTN_OK;
+        }
+        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+    }
     if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
         // key splits: enough CTAs to cover the SMs about twice, never more splits than 128-key tiles
         const int tiles = (d.T_max + 127) / 128;

@@ -1,0 +1,290 @@
+// Step (d) (Eq. 7-8) for up to 64 listed rows of one unit, as a CTA-wide routine on tcgen05.
+//
+// Work is cut into pairs of 128-key tiles.  Two warpgroups alternate over the pairs; inside a
+// warpgroup lanes 0-15 of every warp work on the first tile of the pair and lanes 16-31 on the
+// second one: tcgen05.mma with M = 64 puts row m of its accumulator in TMEM lane
+// (m mod 16) + 32 * (m / 16), so two such accumulators interleave in one column range (the second
+// at lane offset 16) and one tcgen05.ld serves both.  Per pair and warpgroup:
+//   control thread   TMA K pair, V pair -> shared memory (128-byte swizzle)
+//   control thread   S_a = Q K_a^T, S_b = Q K_b^T -> TMEM
+//   warpgroup        masked online softmax of (row, tile) per thread; P_a, P_b (bf16) -> shared memory
+//   control thread   O_a = P_a V_a, O_b = P_b V_b -> TMEM
+//   warpgroup        acc = acc * alpha + O
+// The control thread is a small polling scheduler so that neither warpgroup waits for the other.
+// At the end the (m, l, acc) states of the two tiles of a pair and of the two warpgroups are merged.
+// Every wait is bounded; on expiry the routine sets the status bit and unwinds.
+#pragma once
+#include "psattn_common.cuh"
+#include "psattn_sm100.cuh"
+
+namespace psattn {
+
+constexpr uint32_t kA64Tile = 16384;                         // one 128-key K or V tile
+constexpr uint32_t kA64OffQ = 0;                             // 64 rows x 128 B
+constexpr uint32_t kA64OffWg = 8192;                         // per warpgroup: K pair, V pair, P pair
+constexpr uint32_t kA64WgBytes = 6 * kA64Tile;
+constexpr uint32_t kA64OffBar = kA64OffWg + 2 * kA64WgBytes;
+constexpr uint32_t kA64Bytes = kA64OffBar + 128;
+constexpr uint32_t kA64TmemCols = 512;                       // per warpgroup: S 128 columns, O 64 columns
+constexpr int kA64MaxRows = 64;
+
+struct Attend64Job {
+    int b, h, L;                 // unit and its valid length
+    int lo, hi;                  // key range of this CTA (lo a multiple of 128 relative to 0)
+    const int *rows;             // listed positions (global or shared), or null = identity
+    int n_rows;                  // <= 64
+    int pos_t, pos_h, pos_b;     // TMA coordinate slots
+    int ctrl_warp, wg_warp0;     // warp of the control thread; first warp of warpgroup 0 (multiple of 4)
+};
+
+// All threads of the CTA call this (it contains __syncthreads).  On return the threads of
+// warpgroup 0 with lane < 16 hold, for row 16 * (warp - wg_warp0) + lane, the softmax state over
+// [lo, hi): m (scaled log2 units), l, acc[64] (unnormalised).  Returns false if a wait expired.
+__device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, const Geom &g,
+                                             const Attend64Job &j, const __nv_bfloat16 *__restrict__ Q,
+                                             const CUtensorMap *tmK, const CUtensorMap *tmV, float &m_out,
+                                             float &l_out, float acc[kD]) {
+    using namespace sm100;
+    uint64_t *kfull = reinterpret_cast<uint64_t *>(smem + kA64OffBar);   // [2] per warpgroup
+    uint64_t *vfull = kfull + 2, *sfull = kfull + 4, *pready = kfull + 6, *ofull = kfull + 8;
+    volatile uint32_t *abort_flag = reinterpret_cast<uint32_t *>(kfull + 10);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_tiles = (j.hi - j.lo + 127) / 128, n_pairs = (n_tiles + 1) / 2;
+
+    if (tid == 0) {
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&kfull[x], 1); mbar_init(&vfull[x], 1); mbar_init(&sfull[x], 1);
+            mbar_init(&pready[x], 128); mbar_init(&ofull[x], 1);
+        }
+        *abort_flag = 0u;
+        fence_barrier_init();
+    }
+    // Q rows -> shared memory, K-major, 128-byte swizzle; unused rows are zero
+    for (int e = tid; e < kA64MaxRows * 8; e += blockDim.x) {
+        const int r = e >> 3, c = e & 7;
+        int i = -1;
+        if (r < j.n_rows) i = j.rows ? j.rows[r] : r;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i >= 0 && i < j.L)
+            v = __ldg(reinterpret_cast<const uint4 *>(Q + unit_off(g.qs, j.b, j.h) + (long long)i * g.qs[2]) + c);
+        *reinterpret_cast<uint4 *>(smem + kA64OffQ + r * 128 + ((c ^ (r & 7)) << 4)) = v;
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    const float kScaleLog2 = kScale * kLog2e;
+    float m_run = -INFINITY, l_run = 0.f;
+#pragma unroll
+    for (int c = 0; c < kD; ++c) acc[c] = 0.f;
+
+    if (warp == j.ctrl_warp) {
+        if (lane == 0 && n_pairs > 0) {
+            // ------------------------------ control thread ------------------------------------------
+            constexpr uint32_t kIdescS = umma_idesc_bf16(64, 128, 0);       // B = K tile, K-major
+            constexpr uint32_t kIdescO = umma_idesc_bf16(64, kD, 1);        // B = V tile, MN-major
+            auto coords = [&](int tile, int &c1, int &c2, int &c3) {
+                const int key0 = j.lo + tile * 128;
+                c1 = j.pos_t == 1 ? key0 : (j.pos_h == 1 ? j.h : j.b);
+                c2 = j.pos_t == 2 ? key0 : (j.pos_h == 2 ? j.h : j.b);
+                c3 = j.pos_t == 3 ? key0 : (j.pos_h == 3 ? j.h : j.b);
+            };
+            auto load_pair = [&](int wg, int q, bool is_v) {
+                uint8_t *dst = smem + kA64OffWg + wg * kA64WgBytes + (is_v ? 2 * kA64Tile : 0);
+                uint64_t *bar = is_v ? &vfull[wg] : &kfull[wg];
+                const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
+                mbar_expect_tx(bar, kA64Tile * (1 + two));
+                for (int s = 0; s <= two; ++s) {
+                    int c1, c2, c3;
+                    coords(2 * q + s, c1, c2, c3);
+                    tma_load_4d(dst + s * kA64Tile, is_v ? tmV : tmK, bar, 0, c1, c2, c3);
+                }
+            };
+            int q_of[2] = {0, 1}, stage[2] = {0, 0}, k_pref[2] = {0, 0};
+            for (int wg = 0; wg < 2; ++wg)
+                if (q_of[wg] < n_pairs) { load_pair(wg, q_of[wg], false); load_pair(wg, q_of[wg], true); }
+            const unsigned long long t0 = global_ns();
+            unsigned polls = 0;
+            while ((q_of[0] < n_pairs || q_of[1] < n_pairs) && !*abort_flag) {
+                for (int wg = 0; wg < 2; ++wg) {
+                    const int q = q_of[wg];
+                    if (q >= n_pairs) continue;
+                    const uint32_t ph = (uint32_t)((q >> 1) & 1);
+                    const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
+                    const uint32_t wg_smem = smem_u32(smem + kA64OffWg + wg * kA64WgBytes);
+                    const uint32_t t_s = tmem_base + wg * 192, t_o = t_s + 128;
+                    if (stage[wg] == 0) {
+                        if (mbar_try_wait(&kfull[wg], ph)) {
+                            tc_fence_after();
+                            const uint32_t qa = smem_u32(smem + kA64OffQ);
+                            for (int s = 0; s <= two; ++s)
+#pragma unroll
+                                for (int k = 0; k < kD / 16; ++k)
+                                    umma_bf16(t_s + ((uint32_t)(16 * s) << 16), umma_desc_sw128(qa + k * 32, 16, 1024),
+                                              umma_desc_sw128(wg_smem + s * kA64Tile + k * 32, 16, 1024), kIdescS, k > 0);
+                            umma_commit(&sfull[wg]);
+                            stage[wg] = 1;
+                        }
+                    } else if (stage[wg] == 1) {
+                        if (!k_pref[wg] && q + 2 < n_pairs && mbar_try_wait(&sfull[wg], ph)) {
+                            load_pair(wg, q + 2, false);        // the K buffers are free once S is done
+                            k_pref[wg] = 1;
+                        }
+                        if (mbar_try_wait(&pready[wg], ph) && mbar_try_wait(&vfull[wg], ph)) {
+                            tc_fence_after();
+                            for (int s = 0; s <= two; ++s)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)
+                                    umma_bf16(t_o + ((uint32_t)(16 * s) << 16),
+                                              umma_desc_sw128(wg_smem + (4 + s) * kA64Tile + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024),
+                                              umma_desc_sw128(wg_smem + (2 + s) * kA64Tile + k * 2048, 16, 1024), kIdescO, k > 0);
+                            umma_commit(&ofull[wg]);
+                            stage[wg] = 2;
+                        }
+                    } else {
+                        if (mbar_try_wait(&ofull[wg], ph)) {
+                            if (q + 2 < n_pairs) {
+                                if (!k_pref[wg]) load_pair(wg, q + 2, false);
+                                load_pair(wg, q + 2, true);
+                            }
+                            q_of[wg] = q + 2; k_pref[wg] = 0; stage[wg] = 0;
+                        }
+                    }
+                }
+                if ((++polls & 255u) == 0u && global_ns() - t0 > 2 * kWaitNs) {
+                    *abort_flag = 1u;
+                    atomicOr(g.status, kStatusWaitExpired);
+                }
+            }
+        }
+    } else if (warp >= j.wg_warp0 && warp < j.wg_warp0 + 8) {
+        // ---------------------------------- warpgroups ------------------------------------------------
+        const int wg = (warp - j.wg_warp0) >> 2, w4 = (warp - j.wg_warp0) & 3;
+        const int sub = lane >> 4, row = 16 * w4 + (lane & 15);
+        const bool warp_active = 16 * w4 < j.n_rows;
+        const int wtid = (warp - j.wg_warp0 - 4 * wg) * 32 + lane;          // 0..127 inside the warpgroup
+        uint8_t *wg_smem = smem + kA64OffWg + wg * kA64WgBytes;
+        const uint32_t t_lane = tmem_base + wg * 192 + ((uint32_t)(32 * w4) << 16);
+        uint8_t *prow = wg_smem + (4 + sub) * kA64Tile + row * 128;
+        int cnt = 0;
+        for (int q = wg; q < n_pairs; q += 2, ++cnt) {
+            const uint32_t ph = (uint32_t)(cnt & 1);
+            if (*abort_flag) break;
+            if (!mbar_wait(&sfull[wg], ph)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); break; }
+            tc_fence_after();
+            const int valid_a = min(128, j.hi - (j.lo + 2 * q * 128));
+            const int valid_b = max(0, min(128, j.hi - (j.lo + (2 * q + 1) * 128)));
+            const int valid = sub ? valid_b : valid_a;
+            float alpha = 1.f;
+            __syncwarp();
+            if (warp_active) {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int cb = 0; cb < 8; ++cb) {
+                    float v[16];
+                    tmem_ld16(t_lane + cb * 16, v);
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) if (cb * 16 + x < valid) mx = fmaxf(mx, v[x]);
+                }
+                const float m_new = fmaxf(m_run, mx * kScaleLog2);
+                const float m_use = valid > 0 ? m_new : 0.f;            // an absent tile contributes nothing
+                alpha = valid > 0 ? exp2f(m_run - m_new) : 1.f;         // 0 on a thread's first tile
+                float lsum = 0.f;
+#pragma unroll
+                for (int cb = 0; cb < 8; ++cb) {
+                    float v[16];
+                    tmem_ld16(t_lane + cb * 16, v);
+                    uint32_t packed[8];
+#pragma unroll
+                    for (int x = 0; x < 16; x += 2) {
+                        const float p0 = (cb * 16 + x < valid) ? exp2f(fmaf(v[x], kScaleLog2, -m_use)) : 0.f;
+                        const float p1 = (cb * 16 + x + 1 < valid) ? exp2f(fmaf(v[x + 1], kScaleLog2, -m_use)) : 0.f;
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                        // the weights that multiply V are the rounded ones: sum those for the denominator
+                        lsum += __low2float(pk) + __high2float(pk);
+                        packed[x >> 1] = *reinterpret_cast<uint32_t *>(&pk);
+                    }
+                    // 16 keys = 32 bytes = chunks 2*(cb%4), 2*(cb%4)+1 of panel cb/4
+                    uint8_t *pp = prow + (cb >> 2) * 8192;
+                    const int ch = (cb & 3) * 2;
+                    *reinterpret_cast<uint4 *>(pp + (((ch) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                    *reinterpret_cast<uint4 *>(pp + (((ch + 1) ^ (row & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                }
+                if (valid > 0) { l_run = l_run * alpha + lsum; m_run = m_new; }
+            }
+            // rows of V past the valid length may hold anything (even NaN): zero them so that 0 * x stays 0
+            if (valid_a < 128 || (valid_b > 0 && valid_b < 128)) {          // uniform over the warpgroup
+                if (!mbar_wait(&vfull[wg], ph)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); break; }
+                uint4 *va = reinterpret_cast<uint4 *>(wg_smem + 2 * kA64Tile), *vb = reinterpret_cast<uint4 *>(wg_smem + 3 * kA64Tile);
+                for (int e = valid_a * 8 + wtid; e < 128 * 8; e += 128) va[e] = make_uint4(0u, 0u, 0u, 0u);
+                if (valid_b > 0)
+                    for (int e = valid_b * 8 + wtid; e < 128 * 8; e += 128) vb[e] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(&pready[wg]);
+            if (!mbar_wait(&ofull[wg], ph)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); break; }
+            tc_fence_after();
+            __syncwarp();
+            if (warp_active) {
+#pragma unroll
+                for (int cb = 0; cb < 4; ++cb) {
+                    float v[16];
+                    tmem_ld16(t_lane + 128 + cb * 16, v);
+                    if (valid > 0) {
+#pragma unroll
+                        for (int x = 0; x < 16; ++x) acc[cb * 16 + x] = fmaf(acc[cb * 16 + x], alpha, v[x]);
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+        // merge the two tiles of the pair stream: lanes l and l ^ 16 hold the same row
+        __syncwarp();
+        {
+            const float m_o = __shfl_xor_sync(0xffffffffu, m_run, 16);
+            const float m_new = fmaxf(m_run, m_o);
+            const float f = l_run > 0.f ? exp2f(m_run - m_new) : 0.f;
+            l_run *= f;
+            l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
+#pragma unroll
+            for (int c = 0; c < kD; ++c) {
+                const float x = acc[c] * f;
+                acc[c] = x + __shfl_xor_sync(0xffffffffu, x, 16);
+            }
+            m_run = m_new;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    // merge warpgroup 1 into warpgroup 0 through shared memory (the P area of warpgroup 1 is free now)
+    float *xchg = reinterpret_cast<float *>(smem + kA64OffWg + kA64WgBytes + 4 * kA64Tile);
+    if (warp >= j.wg_warp0 + 4 && warp < j.wg_warp0 + 8 && lane < 16) {
+        const int row = 16 * (warp - j.wg_warp0 - 4) + lane;
+        xchg[row * 66] = m_run; xchg[row * 66 + 1] = l_run;
+#pragma unroll
+        for (int c = 0; c < kD; ++c) xchg[row * 66 + 2 + c] = acc[c];
+    }
+    __syncthreads();
+    if (warp >= j.wg_warp0 && warp < j.wg_warp0 + 4 && lane < 16) {
+        const int row = 16 * (warp - j.wg_warp0) + lane;
+        const float m1 = xchg[row * 66], l1 = xchg[row * 66 + 1];
+        const float m_new = fmaxf(m_run, m1);
+        const float f0 = l_run > 0.f ? exp2f(m_run - m_new) : 0.f, f1 = l1 > 0.f ? exp2f(m1 - m_new) : 0.f;
+        l_run = l_run * f0 + l1 * f1;
+#pragma unroll
+        for (int c = 0; c < kD; ++c) acc[c] = acc[c] * f0 + xchg[row * 66 + 2 + c] * f1;
+        m_run = m_new;
+    }
+    m_out = m_run; l_out = l_run;
+    const bool ok = *abort_flag == 0u;
+    if (!ok && tid == 0) {
+        // copies that were issued but never consumed: give them a bounded chance to land
+        for (int x = 0; x < 2; ++x) { mbar_wait(&kfull[x], 0); mbar_wait(&vfull[x], 0); }
+    }
+    __syncthreads();
+    return ok;
+}
+
+}  // namespace psattn

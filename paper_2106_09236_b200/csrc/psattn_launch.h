@@ -40,6 +40,12 @@ cudaError_t launch_attend_tc(const Geom &g, const void *Q, const void *K, const 
                              int n_rows, int rows_stride, int n_splits, int split_keys, float *part_ml,
                              float *part_acc, void *out, long long out_unit_stride, long long out_row_stride,
                              int out_by_position, int out_fp32, cudaStream_t st);
+// Same step for row lists of at most 64 rows (the sparse path): two warpgroups over pairs of key
+// tiles.  split_keys must be a multiple of 256.  cudaErrorNotSupported: use launch_attend_tc.
+cudaError_t launch_attend64(const Geom &g, const void *Q, const void *K, const void *V, const int *rows,
+                            int n_rows, int rows_stride, int n_splits, int split_keys, float *part_ml,
+                            float *part_acc, void *out, long long out_unit_stride, long long out_row_stride,
+                            int out_by_position, int out_fp32, cudaStream_t st);
 cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows, int n_rows, int rows_stride,
                                 int n_splits, const float *part_ml, const float *part_acc, void *out,
                                 long long out_unit_stride, long long out_row_stride, int out_by_position,

@@ -35,6 +35,8 @@ struct Attend64Job {
     int n_rows;                  // <= 64
     int pos_t, pos_h, pos_b;     // TMA coordinate slots
     int ctrl_warp, wg_warp0;     // warp of the control thread; first warp of warpgroup 0 (multiple of 4)
+    int sum_row;                 // slot (>= n_rows, < 64) whose weights are all 1: it returns the column
+                                 // sums of V over [lo, hi) with l = number of keys; -1 = none
 };
 
 // All threads of the CTA call this (it contains __syncthreads).  On return the threads of
@@ -51,13 +53,33 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_tiles = (j.hi - j.lo + 127) / 128, n_pairs = (n_tiles + 1) / 2;
 
-    if (tid == 0) {
+    auto coords = [&](int tile, int &c1, int &c2, int &c3) {
+        const int key0 = j.lo + tile * 128;
+        c1 = j.pos_t == 1 ? key0 : (j.pos_h == 1 ? j.h : j.b);
+        c2 = j.pos_t == 2 ? key0 : (j.pos_h == 2 ? j.h : j.b);
+        c3 = j.pos_t == 3 ? key0 : (j.pos_h == 3 ? j.h : j.b);
+    };
+    auto load_pair = [&](int wg, int q, bool is_v) {            // control thread only
+        uint8_t *dst = smem + kA64OffWg + wg * kA64WgBytes + (is_v ? 2 * kA64Tile : 0);
+        uint64_t *bar = is_v ? &vfull[wg] : &kfull[wg];
+        const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
+        mbar_expect_tx(bar, kA64Tile * (1 + two));
+        for (int s = 0; s <= two; ++s) {
+            int c1, c2, c3;
+            coords(2 * q + s, c1, c2, c3);
+            tma_load_4d(dst + s * kA64Tile, is_v ? tmV : tmK, bar, 0, c1, c2, c3);
+        }
+    };
+    if (warp == j.ctrl_warp && lane == 0) {
         for (int x = 0; x < 2; ++x) {
             mbar_init(&kfull[x], 1); mbar_init(&vfull[x], 1); mbar_init(&sfull[x], 1);
             mbar_init(&pready[x], 128); mbar_init(&ofull[x], 1);
         }
         *abort_flag = 0u;
         fence_barrier_init();
+        // the first pair of each warpgroup does not depend on the query rows: start it right away
+        for (int wg = 0; wg < 2; ++wg)
+            if (wg < n_pairs) { load_pair(wg, wg, false); load_pair(wg, wg, true); }
     }
     // Q rows -> shared memory, K-major, 128-byte swizzle; unused rows are zero
     for (int e = tid; e < kA64MaxRows * 8; e += blockDim.x) {
@@ -84,26 +106,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             // ------------------------------ control thread ------------------------------------------
             constexpr uint32_t kIdescS = umma_idesc_bf16(64, 128, 0);       // B = K tile, K-major
             constexpr uint32_t kIdescO = umma_idesc_bf16(64, kD, 1);        // B = V tile, MN-major
-            auto coords = [&](int tile, int &c1, int &c2, int &c3) {
-                const int key0 = j.lo + tile * 128;
-                c1 = j.pos_t == 1 ? key0 : (j.pos_h == 1 ? j.h : j.b);
-                c2 = j.pos_t == 2 ? key0 : (j.pos_h == 2 ? j.h : j.b);
-                c3 = j.pos_t == 3 ? key0 : (j.pos_h == 3 ? j.h : j.b);
-            };
-            auto load_pair = [&](int wg, int q, bool is_v) {
-                uint8_t *dst = smem + kA64OffWg + wg * kA64WgBytes + (is_v ? 2 * kA64Tile : 0);
-                uint64_t *bar = is_v ? &vfull[wg] : &kfull[wg];
-                const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
-                mbar_expect_tx(bar, kA64Tile * (1 + two));
-                for (int s = 0; s <= two; ++s) {
-                    int c1, c2, c3;
-                    coords(2 * q + s, c1, c2, c3);
-                    tma_load_4d(dst + s * kA64Tile, is_v ? tmV : tmK, bar, 0, c1, c2, c3);
-                }
-            };
             int q_of[2] = {0, 1}, stage[2] = {0, 0}, k_pref[2] = {0, 0};
-            for (int wg = 0; wg < 2; ++wg)
-                if (q_of[wg] < n_pairs) { load_pair(wg, q_of[wg], false); load_pair(wg, q_of[wg], true); }
             const unsigned long long t0 = global_ns();
             unsigned polls = 0;
             while ((q_of[0] < n_pairs || q_of[1] < n_pairs) && !*abort_flag) {
@@ -115,7 +118,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
                     const uint32_t wg_smem = smem_u32(smem + kA64OffWg + wg * kA64WgBytes);
                     const uint32_t t_s = tmem_base + wg * 192, t_o = t_s + 128;
                     if (stage[wg] == 0) {
-                        if (mbar_try_wait(&kfull[wg], ph)) {
+                        if (mbar_test(&kfull[wg], ph)) {
                             tc_fence_after();
                             const uint32_t qa = smem_u32(smem + kA64OffQ);
                             for (int s = 0; s <= two; ++s)
@@ -127,11 +130,11 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
                             stage[wg] = 1;
                         }
                     } else if (stage[wg] == 1) {
-                        if (!k_pref[wg] && q + 2 < n_pairs && mbar_try_wait(&sfull[wg], ph)) {
+                        if (!k_pref[wg] && q + 2 < n_pairs && mbar_test(&sfull[wg], ph)) {
                             load_pair(wg, q + 2, false);        // the K buffers are free once S is done
                             k_pref[wg] = 1;
                         }
-                        if (mbar_try_wait(&pready[wg], ph) && mbar_try_wait(&vfull[wg], ph)) {
+                        if (mbar_test(&pready[wg], ph) && mbar_test(&vfull[wg], ph)) {
                             tc_fence_after();
                             for (int s = 0; s <= two; ++s)
 #pragma unroll
@@ -143,7 +146,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
                             stage[wg] = 2;
                         }
                     } else {
-                        if (mbar_try_wait(&ofull[wg], ph)) {
+                        if (mbar_test(&ofull[wg], ph)) {
                             if (q + 2 < n_pairs) {
                                 if (!k_pref[wg]) load_pair(wg, q + 2, false);
                                 load_pair(wg, q + 2, true);
@@ -162,7 +165,8 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
         // ---------------------------------- warpgroups ------------------------------------------------
         const int wg = (warp - j.wg_warp0) >> 2, w4 = (warp - j.wg_warp0) & 3;
         const int sub = lane >> 4, row = 16 * w4 + (lane & 15);
-        const bool warp_active = 16 * w4 < j.n_rows;
+        const bool warp_active = 16 * w4 < max(j.n_rows, j.sum_row + 1);
+        const bool is_sum = row == j.sum_row;
         const int wtid = (warp - j.wg_warp0 - 4 * wg) * 32 + lane;          // 0..127 inside the warpgroup
         uint8_t *wg_smem = smem + kA64OffWg + wg * kA64WgBytes;
         const uint32_t t_lane = tmem_base + wg * 192 + ((uint32_t)(32 * w4) << 16);
@@ -179,37 +183,51 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             float alpha = 1.f;
             __syncwarp();
             if (warp_active) {
+                // two passes over the 128 scores of this thread's (row, tile), 64 at a time with both
+                // TMEM loads of a half in flight together
+                uint32_t sv[2][32];
                 float mx = -INFINITY;
 #pragma unroll
-                for (int cb = 0; cb < 8; ++cb) {
-                    float v[16];
-                    tmem_ld16(t_lane + cb * 16, v);
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld32_issue(t_lane + hf * 64, sv[0]);
+                    tmem_ld32_issue(t_lane + hf * 64 + 32, sv[1]);
+                    tmem_ld_wait();
+                    tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
 #pragma unroll
-                    for (int x = 0; x < 16; ++x) if (cb * 16 + x < valid) mx = fmaxf(mx, v[x]);
+                    for (int x = 0; x < 64; ++x)
+                        if (hf * 64 + x < valid) mx = fmaxf(mx, __uint_as_float(sv[x >> 5][x & 31]));
                 }
-                const float m_new = fmaxf(m_run, mx * kScaleLog2);
+                float m_new = fmaxf(m_run, mx * kScaleLog2);
+                if (is_sum) m_new = 0.f;
                 const float m_use = valid > 0 ? m_new : 0.f;            // an absent tile contributes nothing
-                alpha = valid > 0 ? exp2f(m_run - m_new) : 1.f;         // 0 on a thread's first tile
+                alpha = valid > 0 ? fast_exp2(m_run - m_new) : 1.f;     // 0 on a thread's first tile
+                if (is_sum) alpha = 1.f;
                 float lsum = 0.f;
 #pragma unroll
-                for (int cb = 0; cb < 8; ++cb) {
-                    float v[16];
-                    tmem_ld16(t_lane + cb * 16, v);
-                    uint32_t packed[8];
+                for (int hf = 0; hf < 2; ++hf) {
+                    tmem_ld32_issue(t_lane + hf * 64, sv[0]);
+                    tmem_ld32_issue(t_lane + hf * 64 + 32, sv[1]);
+                    tmem_ld_wait();
+                    tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
+                    uint8_t *pp = prow + hf * 8192;                      // panel hf: keys 64 * hf ..
 #pragma unroll
-                    for (int x = 0; x < 16; x += 2) {
-                        const float p0 = (cb * 16 + x < valid) ? exp2f(fmaf(v[x], kScaleLog2, -m_use)) : 0.f;
-                        const float p1 = (cb * 16 + x + 1 < valid) ? exp2f(fmaf(v[x + 1], kScaleLog2, -m_use)) : 0.f;
-                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                        // the weights that multiply V are the rounded ones: sum those for the denominator
-                        lsum += __low2float(pk) + __high2float(pk);
-                        packed[x >> 1] = *reinterpret_cast<uint32_t *>(&pk);
+                    for (int ch = 0; ch < 8; ++ch) {                     // 8 keys = one 16-byte chunk
+                        uint32_t packed[4];
+#pragma unroll
+                        for (int x = 0; x < 8; x += 2) {
+                            const int col = ch * 8 + x;
+                            const float s0 = __uint_as_float(sv[col >> 5][col & 31]);
+                            const float s1 = __uint_as_float(sv[(col + 1) >> 5][(col + 1) & 31]);
+                            float p0 = (hf * 64 + col < valid) ? fast_exp2(fmaf(s0, kScaleLog2, -m_use)) : 0.f;
+                            float p1 = (hf * 64 + col + 1 < valid) ? fast_exp2(fmaf(s1, kScaleLog2, -m_use)) : 0.f;
+                            if (is_sum) { p0 = (hf * 64 + col < valid) ? 1.f : 0.f; p1 = (hf * 64 + col + 1 < valid) ? 1.f : 0.f; }
+                            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                            // the weights that multiply V are the rounded ones: sum those for the denominator
+                            lsum += __low2float(pk) + __high2float(pk);
+                            packed[x >> 1] = *reinterpret_cast<uint32_t *>(&pk);
+                        }
+                        *reinterpret_cast<uint4 *>(pp + ((ch ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     }
-                    // 16 keys = 32 bytes = chunks 2*(cb%4), 2*(cb%4)+1 of panel cb/4
-                    uint8_t *pp = prow + (cb >> 2) * 8192;
-                    const int ch = (cb & 3) * 2;
-                    *reinterpret_cast<uint4 *>(pp + (((ch) ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    *reinterpret_cast<uint4 *>(pp + (((ch + 1) ^ (row & 7)) << 4)) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
                 }
                 if (valid > 0) { l_run = l_run * alpha + lsum; m_run = m_new; }
             }
@@ -228,14 +246,14 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             tc_fence_after();
             __syncwarp();
             if (warp_active) {
+                uint32_t ov[2][32];
+                tmem_ld32_issue(t_lane + 128, ov[0]);
+                tmem_ld32_issue(t_lane + 160, ov[1]);
+                tmem_ld_wait();
+                tmem_ld_fence32(ov[0]); tmem_ld_fence32(ov[1]);
+                if (valid > 0) {
 #pragma unroll
-                for (int cb = 0; cb < 4; ++cb) {
-                    float v[16];
-                    tmem_ld16(t_lane + 128 + cb * 16, v);
-                    if (valid > 0) {
-#pragma unroll
-                        for (int x = 0; x < 16; ++x) acc[cb * 16 + x] = fmaf(acc[cb * 16 + x], alpha, v[x]);
-                    }
+                    for (int x = 0; x < 64; ++x) acc[x] = fmaf(acc[x], alpha, __uint_as_float(ov[x >> 5][x & 31]));
                 }
             }
             tc_fence_before();
@@ -245,7 +263,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
         {
             const float m_o = __shfl_xor_sync(0xffffffffu, m_run, 16);
             const float m_new = fmaxf(m_run, m_o);
-            const float f = l_run > 0.f ? exp2f(m_run - m_new) : 0.f;
+            const float f = l_run > 0.f ? fast_exp2(m_run - m_new) : 0.f;
             l_run *= f;
             l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);
 #pragma unroll
@@ -271,7 +289,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
         const int row = 16 * (warp - j.wg_warp0) + lane;
         const float m1 = xchg[row * 66], l1 = xchg[row * 66 + 1];
         const float m_new = fmaxf(m_run, m1);
-        const float f0 = l_run > 0.f ? exp2f(m_run - m_new) : 0.f, f1 = l1 > 0.f ? exp2f(m1 - m_new) : 0.f;
+        const float f0 = l_run > 0.f ? fast_exp2(m_run - m_new) : 0.f, f1 = l1 > 0.f ? fast_exp2(m1 - m_new) : 0.f;
         l_run = l_run * f0 + l1 * f1;
 #pragma unroll
         for (int c = 0; c < kD; ++c) acc[c] = acc[c] * f0 + xchg[row * 66 + 2 + c] * f1;

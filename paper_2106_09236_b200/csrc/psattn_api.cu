@@ -299,6 +299,15 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
+        cudaError_t e = launch_forward_fused(g, plan->U_max, d.fill_mode == PSATTN_FILL_OWN_V, Q, K, V, sample_idx, O,
+                                             sel_idx, M_out, st);
+        if (e == cudaSuccess) return PSATTN_OK;
+        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+        if (d.path == PSATTN_PATH_FUSED) return PSATTN_ERR_UNSUPPORTED;
+    } else if (d.path == PSATTN_PATH_FUSED) {
+        return PSATTN_ERR_UNSUPPORTED;
+    }
     float *M = M_out ? M_out : ws_at<float>(workspace, plan->off_M);
     if ((rc = run_measure(plan, g, Q, K, sample_idx, M, st)) != PSATTN_OK) return rc;
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));

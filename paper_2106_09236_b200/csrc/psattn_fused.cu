@@ -148,7 +148,7 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
     FusedArgs a;
     a.k_bytes = (uint32_t)measure_k_bytes(g.T);
     a.stage_bytes = (uint32_t)measure_stage_bytes(kFusedThreads, g.idx_cols);
-    size_t phase = (size_t)a.k_bytes + 2 * (size_t)a.stage_bytes;
+    size_t phase = (size_t)a.k_bytes + kMeasureStages * (size_t)a.stage_bytes;
     if (phase < kA64Bytes) phase = kA64Bytes;
     a.off_persist = (uint32_t)((phase + 1023) / 1024 * 1024);
     const size_t smem = a.off_persist + ((5 * (size_t)g.T + 127) / 128) * 128 + sizeof(FusedPersist) + 128;

@@ -7,7 +7,7 @@ namespace psattn {
 
 using namespace sm100;
 
-constexpr int kMeasureThreads = 768;
+constexpr int kMeasureThreads = 384;
 
 struct MeasureMmaArgs {
     int q_slices;               // CTAs per unit
@@ -94,7 +94,7 @@ cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const vo
     if (g.B * g.H == 0) return cudaSuccess;
     const size_t k_bytes = measure_k_bytes(g.T);
     const size_t stage_bytes = measure_stage_bytes(kMeasureThreads, g.idx_cols);
-    const size_t smem = k_bytes + 2 * stage_bytes;
+    const size_t smem = k_bytes + kMeasureStages * stage_bytes;
     if (smem > 225 * 1024 || U_max > kMeasureMaxU || U_max < 1) return cudaErrorNotSupported;
     CUtensorMap tmK;
     int pos[3];

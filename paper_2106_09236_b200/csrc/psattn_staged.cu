@@ -44,21 +44,33 @@ __global__ void __launch_bounds__(256) k_measure(Geom g, const DT *__restrict__ 
             if (my < 0 || my >= L) { atomicOr(g.status, kStatusIdxClamped); my = my < 0 ? 0 : L - 1; }
         }
         const int steps = (min(32, U - base) + 3) >> 2;
-        for (int s = 0; s < steps; ++s) {
-            const int src = s * 4 + grp;
-            const int key = __shfl_sync(0xffffffffu, my, src);
-            const bool active = base + src < U;
-            float kk[8];
-            float part = 0.f;
-            if (active) {
-                load8(Ku + (long long)key * g.ks[2], sub, kk);
+        // four steps (16 sampled keys) at a time, all their row reads in flight together; a lane
+        // without a sample reads row 0 (always valid) and its result is dropped
+        for (int s0 = 0; s0 < steps; s0 += 4) {
+            float kk[4][8], part[4];
+            bool active[4];
 #pragma unroll
-                for (int t = 0; t < 8; ++t) part = fmaf(q[t], kk[t], part);
+            for (int x = 0; x < 4; ++x) {
+                const int src = (s0 + x) * 4 + grp;
+                const int key = __shfl_sync(0xffffffffu, my, src & 31);
+                active[x] = s0 + x < steps && base + src < U;
+                load8(Ku + (long long)(active[x] ? key : 0) * g.ks[2], sub, kk[x]);
             }
-            part += __shfl_xor_sync(0xffffffffu, part, 1);
-            part += __shfl_xor_sync(0xffffffffu, part, 2);
-            part += __shfl_xor_sync(0xffffffffu, part, 4);
-            if (active) measure_push(st, part * kScale);
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                part[x] = 0.f;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) part[x] = fmaf(q[t], kk[x][t], part[x]);
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                part[x] += __shfl_xor_sync(0xffffffffu, part[x], 1);
+                part[x] += __shfl_xor_sync(0xffffffffu, part[x], 2);
+                part[x] += __shfl_xor_sync(0xffffffffu, part[x], 4);
+            }
+#pragma unroll
+            for (int x = 0; x < 4; ++x)
+                if (active[x]) measure_push(st, part[x] * kScale);
         }
     }
 #pragma unroll

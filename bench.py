@@ -97,18 +97,30 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
-def cpu_oracle_timing(w, n_cols, steps=1, warmup=0):
+def cpu_oracle_timing(w, n_cols, steps=None, warmup=0, budget_s=12.0):
+    """Times the CPU oracle (as it stands, all host cores over (batch, head) units) on the whole
+    batch of the workload.  steps=None: one pass to calibrate, then as many passes as fit in about
+    `budget_s` seconds of CPU work."""
     from oracle import psattn_oracle as orc
     inp = wl.make_inputs(w, n_cols)
     cores = orc.max_threads()
     queries = int(inp["lengths"].sum()) * w.H
-    for _ in range(warmup):
+
+    def one():
         orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c, nthreads=cores)
+
+    for _ in range(warmup):
+        one()
+    if steps is None:
+        t0 = time.perf_counter()
+        one()
+        first = time.perf_counter() - t0
+        steps = int(max(1, min(200, budget_s / max(first, 1e-3))))
     t0 = time.perf_counter()
     for _ in range(steps):
-        orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c, nthreads=cores)
+        one()
     dt = (time.perf_counter() - t0) / steps
-    return queries / dt, cores, dt, queries
+    return queries / dt, cores, dt, queries, steps
 
 
 def run_reference(args, w):
@@ -117,9 +129,9 @@ def run_reference(args, w):
         return
     from oracle import psattn_oracle as orc
     n_cols = max(orc.count(w.c, L) for L in range(1, w.T + 1))
-    steps = max(1, min(args.steps, 5))
-    warm = max(0, min(args.warmup, 1))
-    qps, cores, dt, queries = cpu_oracle_timing(w, n_cols, steps, warm)
+    steps = max(1, min(args.steps, 50))
+    warm = max(0, min(args.warmup, 2))
+    qps, cores, dt, queries, _ = cpu_oracle_timing(w, n_cols, steps, warm)
     sample = "whole batch of %s (%d valid queries) per step" % (w.name, queries)
     line = {
         "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus,
@@ -324,9 +336,9 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        qps, cores, dt, q = cpu_oracle_timing(w, n_cols)
+        qps, cores, dt, q, n_pass = cpu_oracle_timing(w, n_cols)
         cpu = {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "whole batch of %s (%d valid queries), one pass, %.2f s" % (w.name, q, dt)}
+               "sample": "whole batch of %s (%d valid queries), %d passes of %.3f s each" % (w.name, q, n_pass, dt)}
 
     if rank == 0:
         line = {

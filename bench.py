@@ -144,13 +144,16 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def time_events(fn, steps, torch):
+def time_events(fn, steps, torch, grouped=False):
     """Runs fn(k) for k in range(steps) between two CUDA events on the current stream."""
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     start.record()
     for k in range(steps):
-        fn(k)
+        if grouped:
+            fn(k, steps)
+        else:
+            fn(k)
     end.record()
     torch.cuda.synchronize()
     return start.elapsed_time(end) / steps      # ms per step
@@ -219,7 +222,8 @@ def main():
     launches_per_step = ps.psattn_launch_count() - l0
 
     def capture(fn):
-        """One CUDA graph per buffer set around fn(set index); None when graphs are switched off."""
+        """CUDA graphs around fn(set index): one per buffer set, plus one that runs all sets in turn
+        (fewer graph launches per timed step).  None when graphs are switched off."""
         if args.no_graph:
             return None
         side = torch.cuda.Stream()
@@ -229,24 +233,39 @@ def main():
                 fn(s)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
-        out = []
+        singles = []
         for s in range(n_sets):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
                 fn(s)
-            out.append(g)
-        return out
+            singles.append(g)
+        group = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(group):
+            for s in range(n_sets):
+                fn(s)
+        return singles, group
 
     def replayer(fn, gs):
-        return (lambda k: gs[k % n_sets].replay()) if gs is not None else fn
+        """k -> runs step k.  With graphs: the group graph replays n_sets consecutive steps when k is
+        a multiple of n_sets and enough steps remain; the tail runs through the single graphs."""
+        if gs is None:
+            return lambda k, total=None: fn(k)
+        singles, group = gs
+
+        def run(k, total=None):
+            if total is None:
+                singles[k % n_sets].replay()
+                return
+            full = (total // n_sets) * n_sets
+            if k < full:
+                if k % n_sets == 0:
+                    group.replay()
+            else:
+                singles[k % n_sets].replay()
+        return run
 
     graphs = capture(step)
-
-    def timed_step(k):
-        if graphs is not None:
-            graphs[k % n_sets].replay()
-        else:
-            step(k)
+    timed_step = replayer(step, graphs)
 
     for k in range(max(args.warmup, 3)):
         timed_step(k)
@@ -255,7 +274,7 @@ def main():
         dist.barrier()
     sampler = ClockSampler(local)
     sampler.start()
-    ms = time_events(timed_step, args.steps, torch)
+    ms = time_events(timed_step, args.steps, torch, grouped=True)
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
@@ -283,8 +302,8 @@ def main():
     r_measure, r_rest = replayer(k_measure, capture(k_measure)), replayer(k_rest, capture(k_rest))
     for k in range(3):
         r_measure(k); r_rest(k)
-    kernel_ms = {"measure(a+b)": time_events(r_measure, nk, torch),
-                 "mean_v+attend+fill(d+e)": time_events(r_rest, nk, torch)}
+    kernel_ms = {"measure(a+b)": time_events(r_measure, nk, torch, grouped=True),
+                 "mean_v+attend+fill(d+e)": time_events(r_rest, nk, torch, grouped=True)}
     peak, peak_kind = measured_peaks()
     units = w.B * w.H
     measure_bytes = units * w.T * w.d * elem * 2 + w.B * w.T * n_cols * 4 + units * w.T * 4

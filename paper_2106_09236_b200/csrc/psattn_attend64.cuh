@@ -35,9 +35,64 @@ struct Attend64Job {
     int n_rows;                  // <= 64
     int pos_t, pos_h, pos_b;     // TMA coordinate slots
     int ctrl_warp, wg_warp0;     // warp of the control thread; first warp of warpgroup 0 (multiple of 4)
-    int sum_row;                 // slot (>= n_rows, < 64) whose weights are all 1: it returns the column
-                                 // sums of V over [lo, hi) with l = number of keys; -1 = none
+    int sum_row;                 // slot (>= n_rows, < 64) kept active although it lists no query: its zero
+                                 // query row gets weight 1 on every key, so it returns the column sums of V
+                                 // over [lo, hi) with l = number of keys; -1 = none
 };
+
+// Masked online softmax of one thread's (row, key tile): two passes over its 128 scores in TMEM,
+// 64 at a time with both loads of a half in flight together; P (bf16) goes to the thread's row of
+// the A-operand tile.  FULL: all 128 keys exist (no masks).  A row whose query is zero gets equal
+// weights exp2(0) = 1 with m = 0, so its accumulator row is the column sum of V and its l the
+// number of keys: that is how the all-ones row works, without any special case here.
+template <bool FULL>
+__device__ __forceinline__ void a64_softmax(uint32_t t_lane, uint8_t *prow, int row, int valid, float &m_run,
+                                            float &l_run, float &alpha) {
+    using namespace sm100;
+    const float kScaleLog2 = kScale * kLog2e;
+    uint32_t sv[2][32];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+        tmem_ld32_issue(t_lane + hf * 64, sv[0]);
+        tmem_ld32_issue(t_lane + hf * 64 + 32, sv[1]);
+        tmem_ld_wait();
+        tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
+#pragma unroll
+        for (int x = 0; x < 64; ++x)
+            if (FULL || hf * 64 + x < valid) mx = fmaxf(mx, __uint_as_float(sv[x >> 5][x & 31]));
+    }
+    const bool any = FULL || valid > 0;                        // an absent tile contributes nothing
+    const float m_new = fmaxf(m_run, mx * kScaleLog2);
+    const float m_use = any ? m_new : 0.f;
+    alpha = any ? fast_exp2(m_run - m_new) : 1.f;              // 0 on a thread's first tile
+    float lsum = 0.f;
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+        tmem_ld32_issue(t_lane + hf * 64, sv[0]);
+        tmem_ld32_issue(t_lane + hf * 64 + 32, sv[1]);
+        tmem_ld_wait();
+        tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
+        uint8_t *pp = prow + hf * 8192;                        // panel hf: keys 64 * hf ..
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {                       // 8 keys = one 16-byte chunk
+            uint32_t packed[4];
+#pragma unroll
+            for (int x = 0; x < 8; x += 2) {
+                const int col = ch * 8 + x;
+                const float s0 = __uint_as_float(sv[col >> 5][col & 31]);
+                const float s1 = __uint_as_float(sv[(col + 1) >> 5][(col + 1) & 31]);
+                const float p0 = (FULL || hf * 64 + col < valid) ? fast_exp2(fmaf(s0, kScaleLog2, -m_use)) : 0.f;
+                const float p1 = (FULL || hf * 64 + col + 1 < valid) ? fast_exp2(fmaf(s1, kScaleLog2, -m_use)) : 0.f;
+                lsum += p0 + p1;
+                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                packed[x >> 1] = *reinterpret_cast<uint32_t *>(&pk);
+            }
+            *reinterpret_cast<uint4 *>(pp + ((ch ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+        }
+    }
+    if (any) { l_run = l_run * alpha + lsum; m_run = m_new; }
+}
 
 // All threads of the CTA call this (it contains __syncthreads).  On return the threads of
 // warpgroup 0 with lane < 16 hold, for row 16 * (warp - wg_warp0) + lane, the softmax state over
@@ -96,7 +151,6 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
     __syncthreads();
     tc_fence_after();
 
-    const float kScaleLog2 = kScale * kLog2e;
     float m_run = -INFINITY, l_run = 0.f;
 #pragma unroll
     for (int c = 0; c < kD; ++c) acc[c] = 0.f;
@@ -166,7 +220,6 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
         const int wg = (warp - j.wg_warp0) >> 2, w4 = (warp - j.wg_warp0) & 3;
         const int sub = lane >> 4, row = 16 * w4 + (lane & 15);
         const bool warp_active = 16 * w4 < max(j.n_rows, j.sum_row + 1);
-        const bool is_sum = row == j.sum_row;
         const int wtid = (warp - j.wg_warp0 - 4 * wg) * 32 + lane;          // 0..127 inside the warpgroup
         uint8_t *wg_smem = smem + kA64OffWg + wg * kA64WgBytes;
         const uint32_t t_lane = tmem_base + wg * 192 + ((uint32_t)(32 * w4) << 16);
@@ -183,53 +236,8 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             float alpha = 1.f;
             __syncwarp();
             if (warp_active) {
-                // two passes over the 128 scores of this thread's (row, tile), 64 at a time with both
-                // TMEM loads of a half in flight together
-                uint32_t sv[2][32];
-                float mx = -INFINITY;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    tmem_ld32_issue(t_lane + hf * 64, sv[0]);
-                    tmem_ld32_issue(t_lane + hf * 64 + 32, sv[1]);
-                    tmem_ld_wait();
-                    tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
-#pragma unroll
-                    for (int x = 0; x < 64; ++x)
-                        if (hf * 64 + x < valid) mx = fmaxf(mx, __uint_as_float(sv[x >> 5][x & 31]));
-                }
-                float m_new = fmaxf(m_run, mx * kScaleLog2);
-                if (is_sum) m_new = 0.f;
-                const float m_use = valid > 0 ? m_new : 0.f;            // an absent tile contributes nothing
-                alpha = valid > 0 ? fast_exp2(m_run - m_new) : 1.f;     // 0 on a thread's first tile
-                if (is_sum) alpha = 1.f;
-                float lsum = 0.f;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    tmem_ld32_issue(t_lane + hf * 64, sv[0]);
-                    tmem_ld32_issue(t_lane + hf * 64 + 32, sv[1]);
-                    tmem_ld_wait();
-                    tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
-                    uint8_t *pp = prow + hf * 8192;                      // panel hf: keys 64 * hf ..
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch) {                     // 8 keys = one 16-byte chunk
-                        uint32_t packed[4];
-#pragma unroll
-                        for (int x = 0; x < 8; x += 2) {
-                            const int col = ch * 8 + x;
-                            const float s0 = __uint_as_float(sv[col >> 5][col & 31]);
-                            const float s1 = __uint_as_float(sv[(col + 1) >> 5][(col + 1) & 31]);
-                            float p0 = (hf * 64 + col < valid) ? fast_exp2(fmaf(s0, kScaleLog2, -m_use)) : 0.f;
-                            float p1 = (hf * 64 + col + 1 < valid) ? fast_exp2(fmaf(s1, kScaleLog2, -m_use)) : 0.f;
-                            if (is_sum) { p0 = (hf * 64 + col < valid) ? 1.f : 0.f; p1 = (hf * 64 + col + 1 < valid) ? 1.f : 0.f; }
-                            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                            // the weights that multiply V are the rounded ones: sum those for the denominator
-                            lsum += __low2float(pk) + __high2float(pk);
-                            packed[x >> 1] = *reinterpret_cast<uint32_t *>(&pk);
-                        }
-                        *reinterpret_cast<uint4 *>(pp + ((ch ^ (row & 7)) << 4)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    }
-                }
-                if (valid > 0) { l_run = l_run * alpha + lsum; m_run = m_new; }
+                if (valid_a == 128 && valid_b == 128) a64_softmax<true>(t_lane, prow, row, 128, m_run, l_run, alpha);
+                else a64_softmax<false>(t_lane, prow, row, valid, m_run, l_run, alpha);
             }
             // rows of V past the valid length may hold anything (even NaN): zero them so that 0 * x stays 0
             if (valid_a < 128 || (valid_b > 0 && valid_b < 128)) {          // uniform over the warpgroup

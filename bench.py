@@ -39,6 +39,33 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of the dominant kernel from the
+# ncu capture summarised under profiles/, valid only while the kernel's sources are unchanged.
+TRAFFIC = {
+    "large_bf16": {"kernel": "k_forward_fused", "bytes": 54027776,
+                   "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
+                   "sources_sha1": "caa9b884986a0bcc10d5018771a567772dc0ff5d"},
+}
+TRAFFIC_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.cuh", "psattn_select.cuh",
+                   "psattn_sm100.cuh", "psattn_common.cuh"]
+
+
+def recorded_traffic(workload):
+    """Bytes per launch from the recorded capture, or None if there is none or the kernel changed."""
+    import hashlib
+    rec = TRAFFIC.get(workload)
+    if rec is None:
+        return None
+    h = hashlib.sha1()
+    try:
+        for f in TRAFFIC_SOURCES:
+            with open(os.path.join(ROOT, "paper_2106_09236_b200", "csrc", f), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    return rec["bytes"] if h.hexdigest() == rec["sources_sha1"] else None
+
+
 def algorithmic_bytes(w, lengths, count, elem):
     """Bytes the method itself must move: Q, K, V read once, O written once, the used part of
     sample_idx (shared by heads), sel_idx, lengths."""
@@ -313,7 +340,9 @@ def main():
         roof_kernel, roof_bytes, roof_ms = "measure (steps a+b)", measure_bytes, kernel_ms["measure(a+b)"]
     achieved = roof_bytes / (roof_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_kind": "of " + peak_kind,
+                "unit": "GB/s", "frac": achieved / peak,
+                "traffic": recorded_traffic(w.name) if launches_per_step == 1 else None,
+                "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": roof_bytes}
     path_gbs = alg_bytes / (ms * 1e-3) / 1e9
 

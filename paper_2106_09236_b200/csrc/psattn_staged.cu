@@ -140,7 +140,15 @@ __global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *
         vbar[(long long)unit * kD + threadIdx.x] = L > 0 ? s / (float)L : 0.f;
     }
     if (M == nullptr) return;                  // mean(V) only
-    block_select([&](int i) { return float_key(Mu[i]); }, L, u, g.u_max, out, scratch);
+    // the routine reads every key several times: keep them in shared memory when they fit
+    __shared__ unsigned keys[kSelectSmemKeys];
+    if (L <= kSelectSmemKeys) {
+        for (int i = threadIdx.x; i < L; i += blockDim.x) keys[i] = float_key(Mu[i]);
+        __syncthreads();
+        block_select([&](int i) { return keys[i]; }, L, u, g.u_max, out, scratch);
+    } else {
+        block_select([&](int i) { return float_key(Mu[i]); }, L, u, g.u_max, out, scratch);
+    }
 }
 
 // ---------------------------------------------------------------------------------------

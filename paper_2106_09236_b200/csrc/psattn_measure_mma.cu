@@ -7,7 +7,7 @@ namespace psattn {
 
 using namespace sm100;
 
-constexpr int kMeasureThreads = 384;
+constexpr int kMeasureThreads = 640;
 
 struct MeasureMmaArgs {
     int q_slices;               // CTAs per unit

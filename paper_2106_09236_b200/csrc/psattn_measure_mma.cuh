@@ -23,7 +23,7 @@ namespace psattn {
 
 constexpr int kMeasureBoxRows = 256;      // K rows per TMA box
 constexpr int kMeasureMaxU = 64;          // four rounds of 16 sampled keys
-constexpr int kMeasureStages = 3;         // staging buffers for Q rows and sample rows (2 blocks in flight)
+constexpr int kMeasureStages = 2;         // staging buffers for Q rows and sample rows (2 blocks in flight)
 
 // The shared-memory reads of the gather are not volatile asm, so that the compiler may interleave
 // independent rounds.  What they read is constant between the two barriers around a staged block;

@@ -363,3 +363,22 @@ def test_argument_errors_are_status_codes():
         ps.Plan(1, 1, 64, idx_cols=3)                # narrower than the rule's U
     del small
     plan.close()
+
+
+def test_forced_fused_path_and_its_limits():
+    """PSATTN_PATH_FUSED runs the one-kernel schedule where it applies and refuses, with a status
+    code, where it does not (fp32 inputs; keys that do not fit in shared memory)."""
+    B, H, T, c = 2, 2, 384, 5.0
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 60, n, "bf16", [384, 201])
+    before = ps.psattn_launch_count()
+    O, sel, M, status = _run_forward(inp, "bf16", c, ps.PSATTN_PATH_FUSED)
+    assert ps.psattn_launch_count() - before == 1          # the whole path was one kernel
+    assert status == 0
+    parity.check_forward(O, sel, M, inp, inp["lengths"], "bf16", c)
+    inp32 = _synth(1, 1, 64, 61, orc.count(c, 64), "fp32")
+    with pytest.raises(ps.PsattnError, match="unsupported"):
+        _run_forward(inp32, "fp32", c, ps.PSATTN_PATH_FUSED)
+    big = _synth(1, 1, 4096, 62, orc.count(c, 4096), "bf16")
+    with pytest.raises(ps.PsattnError, match="unsupported"):
+        _run_forward(big, "bf16", c, ps.PSATTN_PATH_FUSED)

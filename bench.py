@@ -22,6 +22,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2106_09236_b200 import sharding  # noqa: E402
 from paper_2106_09236_b200 import workloads as wl  # noqa: E402
 
 METRIC = "prob-sparse attention queries/s"
@@ -227,7 +228,7 @@ def main():
     n_sets = max(2, int(np.ceil(2.2 * L2_BYTES / per_set)) + 1)
     sets, host_sets, queries_per_step, alg_bytes = [], [], None, None
     for s in range(n_sets):
-        inp = wl.make_inputs(w, n_cols, seed=w.seed + 1000 * rank + 17 * s)
+        inp = wl.make_inputs(w, n_cols, seed=sharding.rank_seed(w.seed, rank, s))
         if s == 0:
             host_sets.append(inp)
             queries_per_step = int(inp["lengths"].sum()) * w.H
@@ -305,9 +306,7 @@ def main():
     clocks = sampler.stop()
     if world > 1:
         dist.barrier()
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+        ms = sharding.max_over_ranks(ms, device="cuda")
     status = plan.psattn_read_status()
     value = queries_per_step * world / (ms * 1e-3)
 
@@ -363,9 +362,7 @@ def main():
             dist.barrier()
         e_ms = time_events(lambda k: plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs), ne, torch)
         if world > 1:
-            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+            e_ms = sharding.max_over_ranks(e_ms, device="cuda")
         h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hl, hi))
         d2h = sum(x.numel() * x.element_size() for x in (hO, hs))
         e2e = {"value": queries_per_step * world / (e_ms * 1e-3), "unit": UNIT,

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(kA64Threads, 1) k_attend64(Geom g, Attend64Arg
     j.lo = min(j.L, split * a.split_keys); j.hi = min(j.L, j.lo + a.split_keys);
     j.rows = a.rows + (long long)unit * a.rows_stride; j.n_rows = a.n_rows;
     j.pos_t = a.pos_t; j.pos_h = a.pos_h; j.pos_b = a.pos_b;
-    j.ctrl_warp = 0; j.wg_warp0 = 4; j.sum_row = -1;
+    j.ctrl_warp = 0; j.wg_warp0 = 4; j.sum_row = -1; j.started = 0;
     float m_run, l_run, acc[kD];
     const bool ok = attend64_run(smem, tmem_base, g, j, Q, &tmK, &tmV, m_run, l_run, acc);
 

@@ -35,10 +35,45 @@ struct Attend64Job {
     int n_rows;                  // <= 64
     int pos_t, pos_h, pos_b;     // TMA coordinate slots
     int ctrl_warp, wg_warp0;     // warp of the control thread; first warp of warpgroup 0 (multiple of 4)
+    int started;                 // attend64_start was already run for this job
     int sum_row;                 // slot (>= n_rows, < 64) kept active although it lists no query: its zero
                                  // query row gets weight 1 on every key, so it returns the column sums of V
                                  // over [lo, hi) with l = number of keys; -1 = none
 };
+
+// Control thread only: initialise the barriers of the routine and start the TMA copies of the first
+// key-tile pair of each warpgroup.  They depend only on the unit and its length, not on the listed
+// rows, so a caller may run this early (set Attend64Job::started) to hide the copy latency behind
+// other work; the shared memory of the routine must be free by then.
+__device__ __forceinline__ void attend64_start(uint8_t *smem, const Attend64Job &j, const CUtensorMap *tmK,
+                                               const CUtensorMap *tmV) {
+    using namespace sm100;
+    uint64_t *kfull = reinterpret_cast<uint64_t *>(smem + kA64OffBar);
+    uint64_t *vfull = kfull + 2, *sfull = kfull + 4, *pready = kfull + 6, *ofull = kfull + 8;
+    volatile uint32_t *abort_flag = reinterpret_cast<uint32_t *>(kfull + 10);
+    const int n_tiles = (j.hi - j.lo + 127) / 128, n_pairs = (n_tiles + 1) / 2;
+    for (int x = 0; x < 2; ++x) {
+        mbar_init(&kfull[x], 1); mbar_init(&vfull[x], 1); mbar_init(&sfull[x], 1);
+        mbar_init(&pready[x], 128); mbar_init(&ofull[x], 1);
+    }
+    *abort_flag = 0u;
+    fence_barrier_init();
+    for (int wg = 0; wg < 2 && wg < n_pairs; ++wg) {
+        for (int is_v = 0; is_v < 2; ++is_v) {
+            uint8_t *dst = smem + kA64OffWg + wg * kA64WgBytes + (is_v ? 2 * kA64Tile : 0);
+            uint64_t *bar = is_v ? &vfull[wg] : &kfull[wg];
+            const int two = (2 * wg + 1 < n_tiles) ? 1 : 0;
+            mbar_expect_tx(bar, kA64Tile * (1 + two));
+            for (int s = 0; s <= two; ++s) {
+                const int key0 = j.lo + (2 * wg + s) * 128;
+                const int c1 = j.pos_t == 1 ? key0 : (j.pos_h == 1 ? j.h : j.b);
+                const int c2 = j.pos_t == 2 ? key0 : (j.pos_h == 2 ? j.h : j.b);
+                const int c3 = j.pos_t == 3 ? key0 : (j.pos_h == 3 ? j.h : j.b);
+                tma_load_4d(dst + s * kA64Tile, is_v ? tmV : tmK, bar, 0, c1, c2, c3);
+            }
+        }
+    }
+}
 
 // Masked online softmax of one thread's (row, key tile): two passes over its 128 scores in TMEM,
 // 64 at a time with both loads of a half in flight together; P (bf16) goes to the thread's row of
@@ -125,17 +160,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             tma_load_4d(dst + s * kA64Tile, is_v ? tmV : tmK, bar, 0, c1, c2, c3);
         }
     };
-    if (warp == j.ctrl_warp && lane == 0) {
-        for (int x = 0; x < 2; ++x) {
-            mbar_init(&kfull[x], 1); mbar_init(&vfull[x], 1); mbar_init(&sfull[x], 1);
-            mbar_init(&pready[x], 128); mbar_init(&ofull[x], 1);
-        }
-        *abort_flag = 0u;
-        fence_barrier_init();
-        // the first pair of each warpgroup does not depend on the query rows: start it right away
-        for (int wg = 0; wg < 2; ++wg)
-            if (wg < n_pairs) { load_pair(wg, wg, false); load_pair(wg, wg, true); }
-    }
+    if (!j.started && warp == j.ctrl_warp && lane == 0) attend64_start(smem, j, tmK, tmV);
     // Q rows -> shared memory, K-major, 128-byte swizzle; unused rows are zero
     for (int e = tid; e < kA64MaxRows * 8; e += blockDim.x) {
         const int r = e >> 3, c = e & 7;

@@ -78,6 +78,17 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     if (M_out != nullptr)
         for (int i = tid; i < g.T; i += kFusedThreads) M_out[(long long)unit * g.T + i] = M_s[i];
 
+    // The attention phase reuses the shared memory of the measure phase, which is free now; its first
+    // K/V tiles depend only on the unit, so their copies start before the selection and land behind it.
+    Attend64Job j;
+    j.b = b; j.h = h; j.L = L; j.lo = 0; j.hi = L;
+    j.rows = P.sel; j.n_rows = u;
+    j.pos_t = a.pos_t; j.pos_h = a.pos_h; j.pos_b = a.pos_b;
+    j.ctrl_warp = 0; j.wg_warp0 = 4;
+    j.sum_row = a.own_v ? -1 : u;
+    j.started = 1;
+    if (ok && L > 0 && tid == 0) attend64_start(smem, j, &tmK, &tmV);
+
     // ---- step (c) -----------------------------------------------------------------------------
     block_select([&](int i) { return float_key(M_s[i]); }, L, u, kA64MaxRows, P.sel, P.select);
     for (int r = tid; r < g.u_max; r += kFusedThreads) {
@@ -89,12 +100,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
 
     // ---- step (d), with the column sums of V riding along ------------------------------------------
     if (ok && L > 0) {
-        Attend64Job j;
-        j.b = b; j.h = h; j.L = L; j.lo = 0; j.hi = L;
-        j.rows = P.sel; j.n_rows = u;
-        j.pos_t = a.pos_t; j.pos_h = a.pos_h; j.pos_b = a.pos_b;
-        j.ctrl_warp = 0; j.wg_warp0 = 4;
-        j.sum_row = a.own_v ? -1 : u;
         float m_run, l_run, acc[kD];
         ok = attend64_run(smem, tmem_base, g, j, Q, &tmK, &tmV, m_run, l_run, acc);
         if (ok && warp >= 4 && warp < 8 && lane < 16) {

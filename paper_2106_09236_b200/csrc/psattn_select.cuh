@@ -11,6 +11,7 @@ struct SelectScratch {
     int wtot_gt[32], wtot_eq[32];
     unsigned prefix;
     int remaining;
+    int done;
 };
 
 // All threads of the block call this with the same arguments (blockDim.x a multiple of 32, <= 1024).
@@ -27,7 +28,7 @@ __device__ __forceinline__ void block_select(KeyFn key_of, int L, int u, int u_m
         __syncthreads();
         return;
     }
-    if (tid == 0) { s.prefix = 0u; s.remaining = u; }
+    if (tid == 0) { s.prefix = 0u; s.remaining = u; s.done = 0; }
     unsigned known = 0u;                                   // key bits fixed so far
     for (int shift = 24; shift >= 0; shift -= 8) {
         if (tid < 256) s.hist[tid] = 0;
@@ -56,12 +57,22 @@ __device__ __forceinline__ void block_select(KeyFn key_of, int L, int u, int u_m
                     if (h[bin] >= r) break;
                     r -= h[bin];
                 }
-                s.prefix = prefix | ((unsigned)(lane * 8 + bin) << shift);
-                s.remaining = r;
+                const unsigned value = prefix | ((unsigned)(lane * 8 + bin) << shift);
+                if (h[bin] == r && value != 0u) {
+                    // every key of this bin is taken: the result is "all keys >= value"; no need to
+                    // resolve the lower bits
+                    s.prefix = value - 1u;
+                    s.remaining = 0;
+                    s.done = 1;
+                } else {
+                    s.prefix = value;
+                    s.remaining = r;
+                }
             }
         }
         known |= 0xffu << shift;
         __syncthreads();
+        if (s.done) break;
     }
     const unsigned tau = s.prefix;
     const int need_eq = s.remaining;                       // positions with key == tau to take, lowest first

@@ -158,11 +158,15 @@ int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const void *K, cons
 int psattn_read_status(psattn_plan_t *plan, void *workspace, void *stream, uint32_t *host_bits);
 
 /* Host-buffer front end.  psattn_plan_enable_host_io allocates, once, device staging for
- * Q, K, V, O, lengths, sample_idx, sel_idx and a workspace inside the plan.
- * psattn_forward_host then copies the HOST arrays in (dense layout, descriptor strides
- * ignored), runs psattn_forward, copies O and sel_idx back and synchronises the stream.
- * lengths may be NULL.  Pinned host memory makes the copies asynchronous and fast; pageable
- * memory works but is slower. */
+ * Q, K, V, O, lengths, sample_idx, sel_idx, a workspace, and one internal copy stream with two
+ * events, all owned by the plan.
+ * psattn_forward_host takes HOST arrays (dense layout, descriptor strides ignored), and returns
+ * with O and sel_idx filled in and both streams idle.  Sequences are independent, so the batch
+ * goes through in chunks (2 by default; the environment variable PSATTN_HOST_CHUNKS = 1..64
+ * overrides it): chunk k is copied in and computed on `stream` while the results of chunk k - 1
+ * are copied out on the internal stream.  lengths may be NULL.  Pinned host memory
+ * makes the copies asynchronous and lets the two directions overlap; pageable memory works but
+ * serialises them. */
 int psattn_plan_enable_host_io(psattn_plan_t *plan);
 int psattn_forward_host(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
                         const int32_t *lengths, const int32_t *sample_idx, void *O,

@@ -3,6 +3,7 @@
 #include "../../include/psattn.h"
 
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -25,6 +26,9 @@ struct psattn_plan {
     bool host_io;
     void *h_Q, *h_K, *h_V, *h_O, *h_ws;
     int *h_len, *h_idx, *h_sel;
+    cudaStream_t h_copy_stream;   // device-to-host copies of finished chunks run here
+    cudaEvent_t h_ev[2];          // [0]: a chunk is finished; [1]: its results have been copied out
+    int b_override;               // > 0: number of sequences of the current (chunked) call
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -160,6 +164,7 @@ extern "C" int psattn_plan_destroy(psattn_plan_t *p) {
     if (p->host_io) {
         cudaFree(p->h_Q); cudaFree(p->h_K); cudaFree(p->h_V); cudaFree(p->h_O); cudaFree(p->h_ws);
         cudaFree(p->h_len); cudaFree(p->h_idx); cudaFree(p->h_sel);
+        cudaStreamDestroy(p->h_copy_stream); cudaEventDestroy(p->h_ev[0]); cudaEventDestroy(p->h_ev[1]);
     }
     delete p;
     return PSATTN_OK;
@@ -188,10 +193,12 @@ static int check_ws(const psattn_plan_t *p, const void *ws, size_t bytes) {
     return PSATTN_OK;
 }
 
+static int plan_b(const psattn_plan_t *p) { return p->b_override > 0 ? p->b_override : p->desc.B; }
+
 static Geom make_geom(const psattn_plan_t *p, const int32_t *lengths, void *ws) {
     Geom g;
     const psattn_desc_t &d = p->desc;
-    g.B = d.B; g.H = d.H; g.T = d.T_max;
+    g.B = plan_b(p); g.H = d.H; g.T = d.T_max;
     g.idx_cols = d.idx_cols; g.idx_per_head = d.idx_per_head;
     g.u_max = p->u_max;
     for (int k = 0; k < 3; ++k) {
@@ -436,6 +443,9 @@ extern "C" int psattn_plan_enable_host_io(psattn_plan_t *plan) {
         }
     }
     PSATTN_CU(cudaMemset(plan->h_ws, 0, 256));
+    PSATTN_CU(cudaStreamCreateWithFlags(&plan->h_copy_stream, cudaStreamNonBlocking));
+    PSATTN_CU(cudaEventCreateWithFlags(&plan->h_ev[0], cudaEventDisableTiming));
+    PSATTN_CU(cudaEventCreateWithFlags(&plan->h_ev[1], cudaEventDisableTiming));
     plan->host_io = true;
     return PSATTN_OK;
 }
@@ -448,13 +458,12 @@ extern "C" int psattn_forward_host(psattn_plan_t *plan, const void *Q, const voi
     psattn_desc_t &d = plan->desc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t es = d.dtype == PSATTN_BF16 ? 2 : 4;
-    const size_t n = (size_t)d.B * d.H * d.T_max * kD * es;
-    const size_t nidx = (size_t)d.B * (d.idx_per_head ? d.H : 1) * d.T_max * d.idx_cols * sizeof(int);
-    const size_t nsel = (size_t)d.B * d.H * plan->u_max * sizeof(int);
-    PSATTN_CU(cudaMemcpyAsync(plan->h_Q, Q, n, cudaMemcpyHostToDevice, st));
-    PSATTN_CU(cudaMemcpyAsync(plan->h_K, K, n, cudaMemcpyHostToDevice, st));
-    PSATTN_CU(cudaMemcpyAsync(plan->h_V, V, n, cudaMemcpyHostToDevice, st));
-    PSATTN_CU(cudaMemcpyAsync(plan->h_idx, sample_idx, nidx, cudaMemcpyHostToDevice, st));
+    // Sequences are independent, so the batch goes through in chunks: while chunk k is copied in and
+    // computed on `stream`, the results of chunk k - 1 travel back on a second stream (PCIe is full
+    // duplex).  All chunks share the one workspace; they are ordered by `stream`.
+    const size_t per_b = (size_t)d.H * d.T_max * kD * es;
+    const size_t idx_b = (size_t)(d.idx_per_head ? d.H : 1) * d.T_max * d.idx_cols * sizeof(int);
+    const size_t sel_b = (size_t)d.H * plan->u_max * sizeof(int);
     if (lengths) PSATTN_CU(cudaMemcpyAsync(plan->h_len, lengths, (size_t)d.B * sizeof(int), cudaMemcpyHostToDevice, st));
     // the staging buffers are dense: run with dense strides whatever the descriptor says
     psattn_desc_t saved = d;
@@ -462,13 +471,38 @@ extern "C" int psattn_forward_host(psattn_plan_t *plan, const void *Q, const voi
     std::memset(d.v_stride, 0, sizeof(d.v_stride)); std::memset(d.o_stride, 0, sizeof(d.o_stride));
     check_strides(d.q_stride, d); check_strides(d.k_stride, d);
     check_strides(d.v_stride, d); check_strides(d.o_stride, d);
-    int rc = psattn_forward(plan, plan->h_Q, plan->h_K, plan->h_V, lengths ? plan->h_len : nullptr,
-                            plan->h_idx, plan->h_O, plan->h_sel, nullptr, plan->h_ws,
-                            plan->ws_bytes, stream);
+    int n_chunks = 2;       // measured: every extra chunk costs ~50 us of copy set-up, more than it hides
+    if (const char *env = std::getenv("PSATTN_HOST_CHUNKS")) { const int v = std::atoi(env); if (v >= 1 && v <= 64) n_chunks = v; }
+    if (n_chunks > d.B) n_chunks = d.B > 0 ? d.B : 1;
+    int rc = PSATTN_OK;
+    cudaError_t ce = cudaSuccess;
+    for (int k = 0; k < n_chunks && rc == PSATTN_OK && ce == cudaSuccess; ++k) {
+        const int b0 = (int)((long long)d.B * k / n_chunks), b1 = (int)((long long)d.B * (k + 1) / n_chunks);
+        const int nb = b1 - b0;
+        if (nb == 0) continue;
+        char *dq = (char *)plan->h_Q + b0 * per_b, *dk = (char *)plan->h_K + b0 * per_b;
+        char *dv = (char *)plan->h_V + b0 * per_b, *dout = (char *)plan->h_O + b0 * per_b;
+        char *di = (char *)plan->h_idx + b0 * idx_b, *ds = (char *)plan->h_sel + b0 * sel_b;
+        if ((ce = cudaMemcpyAsync(dq, (const char *)Q + b0 * per_b, nb * per_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) break;
+        if ((ce = cudaMemcpyAsync(dk, (const char *)K + b0 * per_b, nb * per_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) break;
+        if ((ce = cudaMemcpyAsync(dv, (const char *)V + b0 * per_b, nb * per_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) break;
+        if ((ce = cudaMemcpyAsync(di, (const char *)sample_idx + b0 * idx_b, nb * idx_b, cudaMemcpyHostToDevice, st)) != cudaSuccess) break;
+        plan->b_override = nb;
+        rc = psattn_forward(plan, dq, dk, dv, lengths ? plan->h_len + b0 : nullptr, (const int32_t *)di, dout,
+                            (int32_t *)ds, nullptr, plan->h_ws, plan->ws_bytes, stream);
+        plan->b_override = 0;
+        if (rc != PSATTN_OK) break;
+        if ((ce = cudaEventRecord(plan->h_ev[0], st)) != cudaSuccess) break;
+        if ((ce = cudaStreamWaitEvent(plan->h_copy_stream, plan->h_ev[0], 0)) != cudaSuccess) break;
+        if ((ce = cudaMemcpyAsync((char *)O + b0 * per_b, dout, nb * per_b, cudaMemcpyDeviceToHost, plan->h_copy_stream)) != cudaSuccess) break;
+        if ((ce = cudaMemcpyAsync((char *)sel_idx + b0 * sel_b, ds, nb * sel_b, cudaMemcpyDeviceToHost, plan->h_copy_stream)) != cudaSuccess) break;
+    }
     d = saved;
-    if (rc) return rc;
-    PSATTN_CU(cudaMemcpyAsync(O, plan->h_O, n, cudaMemcpyDeviceToHost, st));
-    PSATTN_CU(cudaMemcpyAsync(sel_idx, plan->h_sel, nsel, cudaMemcpyDeviceToHost, st));
+    plan->b_override = 0;
+    // never return with copies in flight, whatever happened above
+    cudaStreamSynchronize(plan->h_copy_stream);
+    if (rc != PSATTN_OK) { cudaStreamSynchronize(st); return rc; }
+    if (ce != cudaSuccess) { cudaStreamSynchronize(st); return cuda_fail(plan, ce); }
     PSATTN_CU(cudaStreamSynchronize(st));
     return PSATTN_OK;
 }

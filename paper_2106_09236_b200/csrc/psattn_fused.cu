@@ -45,9 +45,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int unit = blockIdx.x, b = unit / g.H, h = unit % g.H;
-    const int L = seq_len(g, b);
-    const int U = min(g.U_tab[L], g.idx_cols);
-    const int u = min(min(g.u_tab[L], g.u_max), L);
     float *M_s = reinterpret_cast<float *>(smem + a.off_persist);
     unsigned char *chosen = reinterpret_cast<unsigned char *>(M_s + g.T);
     FusedPersist &P = *reinterpret_cast<FusedPersist *>(smem + a.off_persist + ((5 * (size_t)g.T + 127) / 128) * 128);
@@ -56,7 +53,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
         if (tid == 0) atomicOr(g.status, kStatusWaitExpired);
         return;
     }
+    // Programmatic dependent launch: let the next kernel of the stream be scheduled already (its CTAs
+    // wait at their own griddepcontrol.wait until this grid has completed and its writes are visible),
+    // and do not touch global memory before the previous grid has completed.  Both are no-ops when the
+    // launch carries no programmatic dependency.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp == 0) tmem_alloc(&P.tmem_slot, kA64TmemCols);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int L = seq_len(g, b);
+    const int U = min(g.U_tab[L], g.idx_cols);
+    const int u = min(min(g.u_tab[L], g.u_max), L);
     if (tid == 32) {
         mbar_init(&P.bar, 1);
         fence_barrier_init();
@@ -173,10 +179,22 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
         if (e != cudaSuccess) return e;
         attr_smem = smem;
     }
-    k_forward_fused<<<(unsigned)(g.B * g.H), kFusedThreads, smem, st>>>(
-        g, a, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)V, sidx, (__nv_bfloat16 *)O, sel, M_out, tmKrows, tmK, tmV);
+    // launched with programmatic stream serialization: the kernel may be scheduled while the previous
+    // kernel of the stream drains; it orders itself with griddepcontrol.wait before its first read
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(g.B * g.H));
+    cfg.blockDim = dim3(kFusedThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_forward_fused, g, a, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)V,
+                                       sidx, (__nv_bfloat16 *)O, sel, M_out, tmKrows, tmK, tmV);
     note_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace psattn

@@ -20,7 +20,7 @@ namespace psattn {
 
 using namespace sm100;
 
-constexpr int kFusedThreads = 384;       // warp 0: control; warps 4-7, 8-11: attention warpgroups
+constexpr int kFusedThreads = 512;       // warp 0: control; warps 4-7, 8-11: attention warpgroups; all 16 warps measure
 
 struct FusedArgs {
     uint32_t k_bytes, stage_bytes;       // measure phase: resident keys, one staging buffer

@@ -229,6 +229,9 @@ static int run_measure(psattn_plan_t *plan, const Geom &g, const void *Q, const 
         cudaError_t e = launch_measure_mma(g, plan->U_max, Q, K, sample_idx, M, st);
         if (e == cudaSuccess) return PSATTN_OK;
         if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+        e = launch_measure_stream(g, plan->U_max, Q, K, sample_idx, M, st);
+        if (e == cudaSuccess) return PSATTN_OK;
+        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
     }
     PSATTN_CU(launch_measure(d.dtype, g, Q, K, sample_idx, M, st));
     return PSATTN_OK;

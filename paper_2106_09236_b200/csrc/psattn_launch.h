@@ -25,6 +25,10 @@ cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const vo
 // cudaErrorNotSupported: shape outside the kernel's limits; run the staged schedule instead.
 cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void *Q, const void *K, const void *V,
                                  const int *sidx, void *O, int *sel, float *M_out, cudaStream_t st);
+// Streaming tensor-datapath form of steps (a)+(b) for bf16 inputs and any T_max (key rows gathered from L2
+// through shared-memory rings); cudaErrorNotSupported when U_max > 64.
+cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
+                                  cudaStream_t st);
 cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, int n_chunks,
                           cudaStream_t st);
 cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,

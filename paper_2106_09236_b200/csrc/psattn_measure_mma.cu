@@ -46,6 +46,32 @@ __global__ void __launch_bounds__(kMeasureThreads, 1) k_measure_mma(Geom g, Meas
                                       sidx, Mu);
 }
 
+// Streaming form (keys gathered from L2 through per-warp rings): any T_max.
+constexpr int kStreamThreads = 512;
+
+__global__ void __launch_bounds__(kStreamThreads, 1) k_measure_stream(Geom g, int q_slices, uint32_t stage_bytes,
+                                                                      const __nv_bfloat16 *__restrict__ Q,
+                                                                      const __nv_bfloat16 *__restrict__ K,
+                                                                      const int *__restrict__ sidx,
+                                                                      float *__restrict__ M) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x;
+    const int unit = blockIdx.x / q_slices, slice = blockIdx.x % q_slices;
+    const int b = unit / g.H, h = unit % g.H;
+    const int L = seq_len(g, b);
+    const int U = min(g.U_tab[L], g.idx_cols);
+    // slices in whole staged blocks so that every CTA but the last works on full blocks
+    constexpr int kBlock = measure_block_queries(kStreamThreads);
+    const int blocks_total = (g.T + kBlock - 1) / kBlock;
+    const int per = (blocks_total + q_slices - 1) / q_slices * kBlock;
+    const int q_lo = min(g.T, slice * per), q_hi = min(g.T, q_lo + per);
+    const int q_end = min(q_hi, L);
+    float *Mu = M + (long long)unit * g.T;
+    for (int i = max(q_lo, L) + tid; i < q_hi; i += kStreamThreads) Mu[i] = 0.f;   // padded queries
+    if (L == 0 || q_lo >= L) return;
+    measure_stream<kStreamThreads>(smem, stage_bytes, g, unit, b, h, L, U, q_lo, q_end, Q, K, sidx, Mu);
+}
+
 // ---- host side ----------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn2)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
@@ -116,6 +142,36 @@ cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const vo
         attr_smem = smem;
     }
     k_measure_mma<<<(unsigned)(units * slices), kMeasureThreads, smem, st>>>(g, a, (const __nv_bfloat16 *)Q, sidx, M, tmK);
+    note_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace psattn
+
+namespace psattn {
+
+// cudaErrorNotSupported: more than 64 samples per query.
+cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
+                                  cudaStream_t st) {
+    if (g.B * g.H == 0) return cudaSuccess;
+    if (U_max > kMeasureMaxU || U_max < 1) return cudaErrorNotSupported;
+    const size_t stage_bytes = measure_stage_bytes(kStreamThreads, g.idx_cols);
+    const size_t smem = (size_t)(kStreamThreads / 32) * kStreamRing * kStreamRoundBytes + 2 * stage_bytes;
+    if (smem > 225 * 1024) return cudaErrorNotSupported;
+    const int units = g.B * g.H;
+    constexpr int kBlock = measure_block_queries(kStreamThreads);
+    const int blocks_total = (g.T + kBlock - 1) / kBlock;
+    int slices = (2 * 148 + units - 1) / units;             // about two CTAs' worth of work per SM
+    if (slices > blocks_total) slices = blocks_total;
+    if (slices < 1) slices = 1;
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        cudaError_t e = cudaFuncSetAttribute(k_measure_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_smem = smem;
+    }
+    k_measure_stream<<<(unsigned)(units * slices), kStreamThreads, smem, st>>>(
+        g, slices, (uint32_t)stage_bytes, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, sidx, M);
     note_launch();
     return cudaGetLastError();
 }

@@ -180,6 +180,147 @@ __device__ __forceinline__ void measure_block(const MeasureCtx &cx) {
         cx.out[q0 + g] = fmaxf((mx - ds / (float)cx.U) * kScale, 0.f);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Streaming form for sequences whose keys do not fit in shared memory: the same eight-queries-per-
+// warp gather-dot, but the 16 sampled key rows of a round are first copied from global memory (L2)
+// into a small per-warp ring in shared memory with cp.async (16 bytes per lane, four copies per
+// round), several rounds ahead.  Random 128-byte row reads out of L2 run far faster than a warp can
+// unpack and multiply them with ordinary instructions, so the arithmetic stays on the tensor-core
+// datapath here too.  Every pair costs one L2 row read, one shared-memory write and one read.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStreamRing = 4;                                  // rounds in flight per warp
+constexpr uint32_t kStreamRoundBytes = 16 * 128;
+
+struct StreamCtx {
+    uint32_t ring;                        // shared-memory address of this warp's ring
+    uint32_t q_tile, idx_tile;            // staged Q rows and sample rows of the block
+    int rows, U, L, idx_cols;
+    uint32_t epoch0;                      // see ldmatrix_x4: produced after the barrier that published the block
+    const __nv_bfloat16 *Ku;              // key rows of the unit
+    long long k_row_stride;               // elements
+    float *out;
+    unsigned *status;
+};
+
+template <int THREADS>
+__device__ __forceinline__ void measure_stream_block(const StreamCtx &cx) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int l7 = lane & 7;
+    const int q0 = warp * 8;
+    if (q0 >= cx.rows) return;
+    const int qn = min(q0 + l7, cx.rows - 1);
+    uint32_t bq[8];
+    {
+        const uint32_t qa = cx.q_tile + (uint32_t)qn * 128u;
+        ldmatrix_x4(qa + ((uint32_t)(((lane >> 3) + l7) & 7) << 4), cx.epoch0, bq[0], bq[1], bq[2], bq[3]);
+        ldmatrix_x4(qa + ((uint32_t)(((lane >> 3) + l7 + 4) & 7) << 4), cx.epoch0, bq[4], bq[5], bq[6], bq[7]);
+    }
+    uint32_t off[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) off[t] = (uint32_t)((2 * t + (lane >> 4) + l7) & 7) << 4;
+    const int slot = (lane >> 3) & 1;                          // this lane's A row is (query l7, sample 2r + slot)
+    const uint32_t krow = cx.idx_tile + (uint32_t)(qn * cx.idx_cols) * 4u;
+    const uint32_t a_row_off = (uint32_t)(l7 + 8 * slot) * 128u;
+    const int g = lane >> 2;
+    const bool de = g & 1;
+    const int rounds = (cx.U + 1) >> 1;
+
+    // copy the 16 key rows of round r into ring stage r % kStreamRing; always commits a group
+    auto issue = [&](int r) {
+        if (r < rounds) {
+            int sample = 2 * r + slot;
+            if (sample >= cx.U) sample = cx.U - 1;             // odd U: the last round repeats its only sample
+            int key = lds_b32(krow + (uint32_t)sample * 4u, cx.epoch0 + (uint32_t)r);
+            if ((unsigned)key >= (unsigned)cx.L) { atomicOr(cx.status, kStatusIdxClamped); key = key < 0 ? 0 : cx.L - 1; }
+            const uint32_t dst = cx.ring + (uint32_t)(r % kStreamRing) * kStreamRoundBytes + (uint32_t)lane * 16u;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int row_e = (lane >> 3) + 4 * k;         // copy e = lane + 32k: row e / 8, chunk e % 8
+                const int key_e = __shfl_sync(0xffffffffu, key, (row_e & 7) + 8 * (row_e >> 3));
+                cp_async_16(dst + (uint32_t)k * 512u, cx.Ku + (long long)key_e * cx.k_row_stride + l7 * 8);
+            }
+        }
+        cp_async_commit();
+    };
+    for (int r = 0; r < kStreamRing - 1; ++r) issue(r);
+
+    float ref = 0.f, mx = 0.f, ds = 0.f;
+    for (int r = 0; r < rounds; ++r) {
+        issue(r + kStreamRing - 1);                            // its stage was read in round r - 1
+        cp_async_wait<kStreamRing - 1>();                      // round r has landed (this lane's copies)
+        __syncwarp();                                          // ... and everybody else's
+        uint32_t epoch;
+        asm volatile("mov.u32 %0, %1;" : "=r"(epoch) : "r"(r) : "memory");
+        float c[4];
+        measure_round(c, cx.ring + (uint32_t)(r % kStreamRing) * kStreamRoundBytes + a_row_off, off, bq, epoch);
+        const float s_lo = de ? c[1] : c[0], s_hi = de ? c[3] : c[2];
+        if (r == 0) ref = s_lo;
+        const float d_lo = s_lo - ref, d_hi = s_hi - ref;
+        const bool hi_ok = 2 * r + 1 < cx.U;
+        mx = fmaxf(mx, fmaxf(d_lo, hi_ok ? d_hi : d_lo));
+        ds += d_lo + (hi_ok ? d_hi : 0.f);
+        __syncwarp();                                          // all reads of this stage are done
+    }
+    cp_async_wait<0>();
+    if ((lane & 3) == (g >> 1) && q0 + g < cx.rows)
+        cx.out[q0 + g] = fmaxf((mx - ds / (float)cx.U) * kScale, 0.f);
+}
+
+// All THREADS threads of the CTA: M~ of the queries [q_lo, q_end) (q_end <= L, L >= 1) of unit (b, h)
+// into out[i].  Shared memory: THREADS / 32 rings, then two staging buffers of stage_bytes.
+// Contains __syncthreads.
+template <int THREADS>
+__device__ __forceinline__ void measure_stream(uint8_t *smem, uint32_t stage_bytes, const Geom &g, int unit, int b, int h,
+                                               int L, int U, int q_lo, int q_end, const __nv_bfloat16 *__restrict__ Q,
+                                               const __nv_bfloat16 *__restrict__ K, const int *__restrict__ sidx,
+                                               float *out) {
+    using namespace sm100;
+    constexpr int kBlock = measure_block_queries(THREADS);
+    constexpr uint32_t kRingBytes = (THREADS / 32) * kStreamRing * kStreamRoundBytes;
+    const int tid = threadIdx.x;
+    const int *idx_base = sidx + ((g.idx_per_head ? (long long)unit : (long long)b) * g.T) * g.idx_cols;
+    const __nv_bfloat16 *Qu = Q + unit_off(g.qs, b, h);
+    const uint32_t stage0 = smem_u32(smem) + kRingBytes;
+    const int n_blocks = (q_end - q_lo + kBlock - 1) / kBlock;
+    auto stage_block = [&](int blk) {
+        if (blk < n_blocks) {
+            const int i0 = q_lo + blk * kBlock;
+            const int rows = min(kBlock, q_end - i0);
+            const uint32_t base = stage0 + (uint32_t)(blk & 1) * stage_bytes;
+            for (int e = tid; e < rows * 8; e += THREADS)
+                cp_async_16(base + (uint32_t)e * 16u, Qu + (long long)(i0 + (e >> 3)) * g.qs[2] + (e & 7) * 8);
+            const int words = rows * g.idx_cols;
+            const int *src = idx_base + (long long)i0 * g.idx_cols;
+            if (((reinterpret_cast<uintptr_t>(src) | (uintptr_t)(words * 4)) & 15u) == 0u) {
+                for (int w = tid; w < words / 4; w += THREADS)
+                    cp_async_16(base + kBlock * 128u + (uint32_t)w * 16u, src + 4 * w);
+            } else {
+                for (int w = tid; w < words; w += THREADS) cp_async_4(base + kBlock * 128u + (uint32_t)w * 4u, src + w);
+            }
+        }
+        cp_async_commit();
+    };
+    StreamCtx cx;
+    cx.ring = smem_u32(smem) + (uint32_t)(tid >> 5) * kStreamRing * kStreamRoundBytes;
+    cx.U = min(U, kMeasureMaxU); cx.L = L; cx.idx_cols = g.idx_cols; cx.status = g.status;
+    cx.Ku = K + unit_off(g.ks, b, h); cx.k_row_stride = g.ks[2];
+    stage_block(0);
+    for (int blk = 0; blk < n_blocks; ++blk) {
+        cp_async_wait<0>();                                    // block blk (and nothing else) is pending
+        __syncthreads();
+        asm volatile("mov.u32 %0, %1;" : "=r"(cx.epoch0) : "r"(blk << 8) : "memory");
+        stage_block(blk + 1);                                  // lands while this block is worked on
+        cx.q_tile = stage0 + (uint32_t)(blk & 1) * stage_bytes;
+        cx.idx_tile = cx.q_tile + kBlock * 128u;
+        const int i0 = q_lo + blk * kBlock;
+        cx.rows = min(kBlock, q_end - i0);
+        cx.out = out + i0;
+        measure_stream_block<THREADS>(cx);
+        __syncthreads();                                       // buffer blk & 1 may be restaged next time
+    }
+    cp_async_wait<0>();
+}
+
 // One thread: start the TMA copies of the unit's key rows [0, L) into shared memory at `smem`
 // (row pitch 128 B), all arriving on `bar` (initialised, count 1).  Returns the number of boxes.
 __device__ __forceinline__ int measure_issue_keys(uint8_t *smem, uint64_t *bar, const CUtensorMap *tmK, int L, int b,

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(kMeasureThreads, 1) k_measure_mma(Geom g, Meas
 }
 
 // Streaming form (keys gathered from L2 through per-warp rings): any T_max.
-constexpr int kStreamThreads = 512;
+constexpr int kStreamThreads = 768;
 
 __global__ void __launch_bounds__(kStreamThreads, 1) k_measure_stream(Geom g, int q_slices, uint32_t stage_bytes,
                                                                       const __nv_bfloat16 *__restrict__ Q,

@@ -188,7 +188,7 @@ __device__ __forceinline__ void measure_block(const MeasureCtx &cx) {
 // unpack and multiply them with ordinary instructions, so the arithmetic stays on the tensor-core
 // datapath here too.  Every pair costs one L2 row read, one shared-memory write and one read.
 // ---------------------------------------------------------------------------------------------
-constexpr int kStreamRing = 4;                                  // rounds in flight per warp
+constexpr int kStreamRing = 2;                                  // rounds in flight per warp
 constexpr uint32_t kStreamRoundBytes = 16 * 128;
 
 struct StreamCtx {

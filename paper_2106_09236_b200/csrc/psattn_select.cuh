@@ -9,6 +9,7 @@ namespace psattn {
 struct SelectScratch {
     int hist[256];
     int wtot_gt[32], wtot_eq[32];
+    int wpre_gt[33], wpre_eq[33];
     unsigned prefix;
     int remaining;
     int done;
@@ -90,12 +91,19 @@ __device__ __forceinline__ void block_select(KeyFn key_of, int L, int u, int u_m
         }
         if (lane == 31) { s.wtot_gt[wid] = xg; s.wtot_eq[wid] = xe; }
         __syncthreads();
-        int bg = 0, be = 0, tg = 0, te = 0;
-        for (int w = 0; w < nw; ++w) {
-            const int a = s.wtot_gt[w], e = s.wtot_eq[w];
-            if (w < wid) { bg += a; be += e; }
-            tg += a; te += e;
+        if (wid == 0) {                                        // exclusive scan of the warp totals; grand totals in [nw]
+            int tg = lane < nw ? s.wtot_gt[lane] : 0, te = lane < nw ? s.wtot_eq[lane] : 0;
+            const int og = tg, oe = te;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int yg = __shfl_up_sync(0xffffffffu, tg, o), ye = __shfl_up_sync(0xffffffffu, te, o);
+                if (lane >= o) { tg += yg; te += ye; }
+            }
+            s.wpre_gt[lane] = tg - og; s.wpre_eq[lane] = te - oe;
+            if (lane == 31) { s.wpre_gt[32] = tg; s.wpre_eq[32] = te; }
         }
+        __syncthreads();
+        const int bg = s.wpre_gt[wid], be = s.wpre_eq[wid], tg = s.wpre_gt[32], te = s.wpre_eq[32];
         const int gt_before = gt_seen + bg + xg - is_gt, eq_before = eq_seen + be + xe - is_eq;
         // taken positions before this one: all greater ones, and the equal ones up to need_eq
         if (is_gt || (is_eq && eq_before < need_eq)) {

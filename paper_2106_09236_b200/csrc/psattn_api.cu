@@ -150,8 +150,9 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     p->off_M = off;      off = align_up(off + units * d.T_max * sizeof(float), 256);
     p->off_vpart = off;  off = align_up(off + units * p->n_chunks * kD * sizeof(float), 256);
     p->off_vbar = off;   off = align_up(off + units * kD * sizeof(float), 256);
-    p->off_ml = off;     off = align_up(off + units * u_max * p->n_splits * 2 * sizeof(float), 256);
-    p->off_acc = off;    off = align_up(off + units * u_max * p->n_splits * kD * sizeof(float), 256);
+    // split partials: u_max row slots per unit plus one for the all-ones row that yields mean(V)
+    p->off_ml = off;     off = align_up(off + units * (u_max + 1) * p->n_splits * 2 * sizeof(float), 256);
+    p->off_acc = off;    off = align_up(off + units * (u_max + 1) * p->n_splits * kD * sizeof(float), 256);
     p->off_sel = off;    off = align_up(off + units * u_max * sizeof(int), 256);
     p->ws_bytes = off;
     *out = p;
@@ -241,10 +242,13 @@ static int run_measure(psattn_plan_t *plan, const Geom &g, const void *Q, const 
 // staged SIMT schedule or the layout has no tensor map), SIMT kernel otherwise.
 static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K, const void *V,
                       const int *rows, int n_rows, int rows_stride, void *out, long long ous,
-                      long long ors, int by_pos, int out_fp32, void *ws, cudaStream_t st) {
+                      long long ors, int by_pos, int out_fp32, void *ws, cudaStream_t st,
+                      float *vbar = nullptr) {
+    // vbar != nullptr: the caller has checked attend64_supported(..., with_vbar = 1); mean(V) comes out of
+    // the attention kernel (an extra all-ones weight row) instead of a separate pass over V
     const psattn_desc_t &d = plan->desc;
     float *ml = ws_at<float>(ws, plan->off_ml), *acc = ws_at<float>(ws, plan->off_acc);
-    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && rows != nullptr && n_rows <= 64) {
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && rows != nullptr && n_rows + (vbar ? 1 : 0) <= 64) {
         // one CTA per SM: split the keys only when there are fewer units than SMs
         const int pairs = (d.T_max + 255) / 256;
         int splits = 148 / (d.B * d.H > 0 ? d.B * d.H : 1);
@@ -254,14 +258,14 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
         const int split_keys = ((pairs + splits - 1) / splits) * 256;
         splits = (d.T_max + split_keys - 1) / split_keys;
         cudaError_t e = launch_attend64(g, Q, K, V, rows, n_rows, rows_stride, splits, split_keys, ml, acc, out, ous,
-                                        ors, by_pos, out_fp32, st);
+                                        ors, by_pos, out_fp32, vbar, st);
         if (e == cudaSuccess) {
             if (splits > 1)
                 PSATTN_CU(merge_attend_splits(!out_fp32, g, rows, n_rows, rows_stride, splits, ml, acc, out, ous,
-                                              ors, by_pos, st));
+                                              ors, by_pos, vbar, st));
             return PSATTN_OK;
         }
-        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+        if (e != cudaErrorNotSupported || vbar != nullptr) return cuda_fail(plan, e);
     }
     if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
         // key splits: enough CTAs to cover the SMs about twice, never more splits than 128-key tiles
@@ -278,7 +282,7 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
         if (e == cudaSuccess) {
             if (splits > 1)
                 PSATTN_CU(merge_attend_splits(!out_fp32, g, rows, n_rows, rows_stride, splits, ml, acc, out, ous,
-                                              ors, by_pos, st));
+                                              ors, by_pos, nullptr, st));
             return PSATTN_OK;
         }
         if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
@@ -289,13 +293,30 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
     return PSATTN_OK;
 }
 
-// Steps (d)+(e) for a selection that already sits in `sel` (device) with vbar in the workspace.
-static int run_attend_and_fill(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K,
-                               const void *V, const int *sel, void *O, void *ws, cudaStream_t st) {
+// Can mean(V) come out of the attention kernel for this plan and these buffers (bf16, at most 63 rows,
+// tensor maps exist, fill value is mean(V))?  Then no separate column-sum pass over V is needed.
+static bool vbar_from_attention(const psattn_plan_t *plan, const Geom &g, const void *K, const void *V) {
     const psattn_desc_t &d = plan->desc;
-    PSATTN_CU(launch_fill(d.dtype, g, V, sel, ws_at<float>(ws, plan->off_vbar), O,
-                          d.fill_mode == PSATTN_FILL_OWN_V, st));
-    return run_attend(plan, g, Q, K, V, sel, plan->u_max, plan->u_max, O, 0, 0, 1, 0, ws, st);
+    return d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && d.fill_mode == PSATTN_FILL_MEAN_V &&
+           attend64_supported(g, K, V, plan->u_max, 1);
+}
+
+// Steps (d)+(e) for a selection that already sits in `sel` (device).  vbar_ready: mean(V) is already
+// in the workspace (column-sum pass); otherwise it is produced by the attention kernel, and the fill
+// runs after it.
+static int run_attend_and_fill(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K,
+                               const void *V, const int *sel, void *O, void *ws, cudaStream_t st,
+                               bool vbar_ready) {
+    const psattn_desc_t &d = plan->desc;
+    float *vbar = ws_at<float>(ws, plan->off_vbar);
+    if (vbar_ready) {
+        PSATTN_CU(launch_fill(d.dtype, g, V, sel, vbar, O, d.fill_mode == PSATTN_FILL_OWN_V, st));
+        return run_attend(plan, g, Q, K, V, sel, plan->u_max, plan->u_max, O, 0, 0, 1, 0, ws, st);
+    }
+    int rc = run_attend(plan, g, Q, K, V, sel, plan->u_max, plan->u_max, O, 0, 0, 1, 0, ws, st, vbar);
+    if (rc != PSATTN_OK) return rc;
+    PSATTN_CU(launch_fill(d.dtype, g, V, sel, vbar, O, 0, st));
+    return PSATTN_OK;
 }
 
 extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
@@ -320,10 +341,14 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
     }
     float *M = M_out ? M_out : ws_at<float>(workspace, plan->off_M);
     if ((rc = run_measure(plan, g, Q, K, sample_idx, M, st)) != PSATTN_OK) return rc;
+    if (vbar_from_attention(plan, g, K, V)) {
+        PSATTN_CU(launch_select(g, M, sel_idx, nullptr, 0, nullptr, st));
+        return run_attend_and_fill(plan, g, Q, K, V, sel_idx, O, workspace, st, false);
+    }
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
     PSATTN_CU(launch_select(g, M, sel_idx, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks,
                             ws_at<float>(workspace, plan->off_vbar), st));
-    return run_attend_and_fill(plan, g, Q, K, V, sel_idx, O, workspace, st);
+    return run_attend_and_fill(plan, g, Q, K, V, sel_idx, O, workspace, st, true);
 }
 
 extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q, const void *K,
@@ -337,12 +362,13 @@ extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
-    // mean(V): column sums, then the finishing part of the select kernel is not needed; use a
-    // select launch with u forced to nothing?  Simpler and exact: the same two kernels.
+    if (vbar_from_attention(plan, g, K, V))
+        return run_attend_and_fill(plan, g, Q, K, V, sel_idx_in, O, workspace, st, false);
+    // mean(V) by a column-sum pass (the select kernel, run without keys, only finishes the mean)
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
     PSATTN_CU(launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart),
                             plan->n_chunks, ws_at<float>(workspace, plan->off_vbar), st));
-    return run_attend_and_fill(plan, g, Q, K, V, sel_idx_in, O, workspace, st);
+    return run_attend_and_fill(plan, g, Q, K, V, sel_idx_in, O, workspace, st, true);
 }
 
 extern "C" int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K,

@@ -54,11 +54,15 @@ cudaError_t launch_attend_tc(const Geom &g, const void *Q, const void *K, const 
 cudaError_t launch_attend64(const Geom &g, const void *Q, const void *K, const void *V, const int *rows,
                             int n_rows, int rows_stride, int n_splits, int split_keys, float *part_ml,
                             float *part_acc, void *out, long long out_unit_stride, long long out_row_stride,
-                            int out_by_position, int out_fp32, cudaStream_t st);
+                            int out_by_position, int out_fp32, float *vbar, cudaStream_t st);
+// With vbar != nullptr launch_attend64 also produces mean(V) [unit][64] (fp32) from an extra row whose
+// weights are all 1, at no extra pass over V; the partials then hold n_rows + 1 row slots per unit.
+bool attend64_supported(const Geom &g, const void *K, const void *V, int n_rows, int with_vbar);
+// vbar != nullptr: the partials hold one more row slot per unit (the all-ones row), merged into vbar.
 cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows, int n_rows, int rows_stride,
                                 int n_splits, const float *part_ml, const float *part_acc, void *out,
                                 long long out_unit_stride, long long out_row_stride, int out_by_position,
-                                cudaStream_t st);
+                                float *vbar, cudaStream_t st);
 cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
                         void *O, int own_v, cudaStream_t st);
 

@@ -259,15 +259,25 @@ __global__ void __launch_bounds__(256) k_attend_combine(Geom g, const int *__res
                                                         OT *__restrict__ out,
                                                         long long out_unit_stride,
                                                         long long out_row_stride,
-                                                        int out_by_position) {
+                                                        int out_by_position, float *__restrict__ vbar) {
+    const int n_slots = n_rows + (vbar ? 1 : 0);           // slot n_rows (if any) is the all-ones row
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long rowid = t / kD;
     const int c = (int)(t % kD);
-    if (rowid >= (long long)g.B * g.H * n_rows) return;
-    const int r = (int)(rowid % n_rows);
-    const int unit = (int)(rowid / n_rows);
+    if (rowid >= (long long)g.B * g.H * n_slots) return;
+    const int r = (int)(rowid % n_slots);
+    const int unit = (int)(rowid / n_slots);
     const int b = unit / g.H, h = unit % g.H;
     const int L = seq_len(g, b);
+    if (r == n_rows) {                                     // mean(V) = merged column sums / merged key count
+        float lw = 0.f, a = 0.f;
+        for (int s = 0; s < n_splits; ++s) {
+            lw += part_ml[2 * (rowid * n_splits + s) + 1];
+            a += part_acc[(rowid * n_splits + s) * kD + c];
+        }
+        vbar[(long long)unit * kD + c] = lw > 0.f ? a / lw : 0.f;
+        return;
+    }
     const int i = rows ? rows[(long long)unit * rows_stride + r] : r;
     const bool row_ok = i >= 0 && i < L;
     OT *dst;
@@ -381,7 +391,7 @@ static cudaError_t launch_attend_t(const Geom &g, const void *Q, const void *K, 
     if (e != cudaSuccess || n_splits == 1) return e;
     const long long threads = (long long)g.B * g.H * n_rows * kD;
     k_attend_combine<OT><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
-        g, rows, n_rows, rows_stride, n_splits, part_ml, part_acc, (OT *)out, ous, ors, by_pos); note_launch();
+        g, rows, n_rows, rows_stride, n_splits, part_ml, part_acc, (OT *)out, ous, ors, by_pos, nullptr); note_launch();
     return cudaGetLastError();
 }
 
@@ -401,18 +411,18 @@ cudaError_t launch_attend_simt(int dtype, int out_fp32, const Geom &g, const voi
 cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows, int n_rows, int rows_stride,
                                 int n_splits, const float *part_ml, const float *part_acc, void *out,
                                 long long out_unit_stride, long long out_row_stride, int out_by_position,
-                                cudaStream_t st) {
-    const long long threads = (long long)g.B * g.H * n_rows * kD;
+                                float *vbar, cudaStream_t st) {
+    const long long threads = (long long)g.B * g.H * (n_rows + (vbar ? 1 : 0)) * kD;
     if (threads == 0) return cudaSuccess;
     const unsigned blocks = (unsigned)((threads + 255) / 256);
     if (out_is_bf16)
         k_attend_combine<__nv_bfloat16><<<blocks, 256, 0, st>>>(g, rows, n_rows, rows_stride, n_splits, part_ml,
                                                                  part_acc, (__nv_bfloat16 *)out, out_unit_stride,
-                                                                 out_row_stride, out_by_position);
+                                                                 out_row_stride, out_by_position, vbar);
     else
         k_attend_combine<float><<<blocks, 256, 0, st>>>(g, rows, n_rows, rows_stride, n_splits, part_ml, part_acc,
                                                         (float *)out, out_unit_stride, out_row_stride,
-                                                        out_by_position);
+                                                        out_by_position, vbar);
     note_launch();
     return cudaGetLastError();
 }

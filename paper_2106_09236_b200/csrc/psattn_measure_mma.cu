@@ -150,11 +150,12 @@ cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const vo
 
 namespace psattn {
 
-// cudaErrorNotSupported: more than 64 samples per query.
+// cudaErrorNotSupported: more than 64 samples per query, or key rows of a unit spread over 4 GB or more.
 cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
                                   cudaStream_t st) {
     if (g.B * g.H == 0) return cudaSuccess;
     if (U_max > kMeasureMaxU || U_max < 1) return cudaErrorNotSupported;
+    if (g.ks[2] <= 0 || (long long)g.T * g.ks[2] * 2 >= (1ll << 32)) return cudaErrorNotSupported;
     const size_t stage_bytes = measure_stage_bytes(kStreamThreads, g.idx_cols);
     const size_t smem = (size_t)(kStreamThreads / 32) * kStreamRing * kStreamRoundBytes + 2 * stage_bytes;
     if (smem > 225 * 1024) return cudaErrorNotSupported;

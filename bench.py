@@ -198,6 +198,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of CUDA-graph replays")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense comparator timing")
+    ap.add_argument("--no-variants", action="store_true",
+                    help="skip the selection-reuse and paper-literal timings")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -330,6 +332,45 @@ def main():
         r_measure(k); r_rest(k)
     kernel_ms = {"measure(a+b)": time_events(r_measure, nk, torch, grouped=True),
                  "mean_v+attend+fill(d+e)": time_events(r_rest, nk, torch, grouped=True)}
+    variants = None
+    if not args.no_variants:
+        variants = {}
+        # Sec. 4.4: N_share consecutive layers share one index set: one full pass, then N_share - 1
+        # passes of steps (d)+(e) on other layers' Q, K, V (the rotating buffer sets stand in for layers)
+        for n_share in (4, 8):
+            def group(k, n=n_share):
+                d0 = sets[(k * n) % n_sets]
+                plan.psattn_forward(d0["Q"], d0["K"], d0["V"], d0["lengths"], d0["sample_idx"], d0["O"], d0["sel"])
+                for j in range(1, n):
+                    d = sets[(k * n + j) % n_sets]
+                    plan.psattn_forward_with_selection(d["Q"], d["K"], d["V"], d["lengths"], d0["sel"], d["O"])
+            r_group = replayer(group, capture(group))
+            for k in range(3):
+                r_group(k)
+            g_ms = time_events(r_group, max(n_sets, nk // n_share), torch, grouped=True)
+            variants["selection_reuse_n_share_%d" % n_share] = {
+                "ms_per_layer": g_ms / n_share, "value": queries_per_step / (g_ms / n_share * 1e-3), "unit": UNIT}
+        # Sec. 3.2 / Eq. 12 as printed: u = ceil(r_sparse * T) selected queries, the others output v_i
+        for r_sparse in (0.35, 0.5):
+            u_lit = int(np.ceil(r_sparse * w.T))
+            plan2 = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, u_override=u_lit,
+                            fill_mode=ps.PSATTN_FILL_OWN_V)
+            sel2 = torch.empty((w.B, w.H, plan2.u_max), dtype=torch.int32, device="cuda")
+
+            def literal(k):
+                d = sets[k % n_sets]
+                plan2.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], sel2)
+            r_lit = replayer(literal, capture(literal))
+            for k in range(3):
+                r_lit(k)
+            l_ms = time_events(r_lit, max(n_sets, min(nk, 50)), torch, grouped=True)
+            flops = 4.0 * w.d * sum(int(L) * min(u_lit, int(L)) for L in host_sets[0]["lengths"]) * w.H
+            variants["paper_literal_r_sparse_%.2f" % r_sparse] = {
+                "u": u_lit, "fill": "own value row", "ms_per_step": l_ms,
+                "value": queries_per_step / (l_ms * 1e-3), "unit": UNIT,
+                "attention_tflops": flops / (l_ms * 1e-3) / 1e12,
+                "device_status": plan2.psattn_read_status()}
+            plan2.close()
     peak, peak_kind = measured_peaks()
     units = w.B * w.H
     measure_bytes = units * w.T * w.d * elem * 2 + w.B * w.T * n_cols * 4 + units * w.T * 4
@@ -400,6 +441,7 @@ def main():
             "path_effective_gbs": path_gbs, "path_frac_of_hbm": path_gbs / peak,
             "algorithmic_bytes_per_step": alg_bytes, "queries_per_step": queries_per_step,
             "kernel_ms": kernel_ms, "direct_call_ms_per_step": direct_ms, "dense": dense,
+            "variants": variants,
             "device_status": status,
         }
         print(json.dumps(line), flush=True)

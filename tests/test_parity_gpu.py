@@ -144,6 +144,23 @@ def test_own_value_fill_and_sample_override(path):
                          fill="own_v")
 
 
+@pytest.mark.parametrize("r_sparse", [0.35, 0.5])
+@pytest.mark.parametrize("dtype,T", [("bf16", 1024), ("fp32", 300)])
+def test_paper_literal_variant_at_scale(dtype, T, r_sparse):
+    """Sec. 3.2's own rule u = ceil(r_sparse * T) (hundreds of selected rows per unit: several
+    128-row tiles of the tensor-core attention and a ragged last one) with Eq. 12's v_i fill."""
+    B, H, c = 2, 4, 5.0
+    lengths = [T, T - 37]
+    u = int(np.ceil(r_sparse * T))
+    n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+    inp = _synth(B, H, T, 146 + T, n_cols, dtype, lengths)
+    O, sel, M, status = _run_forward(inp, dtype, c, ps.PSATTN_PATH_AUTO, u_override=u,
+                                     fill_mode=ps.PSATTN_FILL_OWN_V)
+    assert status == 0
+    assert sel.shape[-1] == u
+    parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c, u_override=u, fill="own_v")
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_out_of_range_inputs_set_status_bits_without_faulting(path):
     B, H, T, c = 2, 1, 80, 5.0

@@ -42,29 +42,38 @@ def measured_peaks():
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of the dominant kernel from the
 # ncu capture summarised under profiles/, valid only while the kernel's sources are unchanged.
-TRAFFIC = {
-    "large_bf16": {"kernel": "k_forward_fused", "bytes": 54027776,
-                   "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
-                   "sources_sha1": "caa9b884986a0bcc10d5018771a567772dc0ff5d"},
-}
-TRAFFIC_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.cuh", "psattn_select.cuh",
+_FUSED_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.cuh", "psattn_select.cuh",
+                  "psattn_sm100.cuh", "psattn_common.cuh"]
+_STREAM_SOURCES = ["psattn_measure_mma.cu", "psattn_measure_stream.cuh", "psattn_measure_mma.cuh",
                    "psattn_sm100.cuh", "psattn_common.cuh"]
+TRAFFIC = {
+    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53704704, "sources": _FUSED_SOURCES,
+                   "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
+                   "sources_sha1": "pending"},
+    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76376576, "sources": _STREAM_SOURCES,
+                  "profile": "profiles/ncu_full_k_measure_stream_long_bf16.txt",
+                  "sources_sha1": "pending"},
+}
+
+
+def sources_sha1(files):
+    import hashlib
+    h = hashlib.sha1()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2106_09236_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
 
 
 def recorded_traffic(workload):
     """Bytes per launch from the recorded capture, or None if there is none or the kernel changed."""
-    import hashlib
     rec = TRAFFIC.get(workload)
     if rec is None:
         return None
-    h = hashlib.sha1()
     try:
-        for f in TRAFFIC_SOURCES:
-            with open(os.path.join(ROOT, "paper_2106_09236_b200", "csrc", f), "rb") as fh:
-                h.update(fh.read())
+        return rec["bytes"] if sources_sha1(rec["sources"]) == rec["sources_sha1"] else None
     except OSError:
         return None
-    return rec["bytes"] if h.hexdigest() == rec["sources_sha1"] else None
 
 
 def algorithmic_bytes(w, lengths, count, elem):
@@ -381,7 +390,7 @@ def main():
     achieved = roof_bytes / (roof_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak,
-                "traffic": recorded_traffic(w.name) if launches_per_step == 1 else None,
+                "traffic": recorded_traffic(w.name),
                 "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": roof_bytes}
     path_gbs = alg_bytes / (ms * 1e-3) / 1e9

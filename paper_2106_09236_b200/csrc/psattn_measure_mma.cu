@@ -2,6 +2,7 @@
 // One CTA = (unit, slice of its queries).
 #include "psattn_launch.h"
 #include "psattn_measure_mma.cuh"
+#include "psattn_measure_stream.cuh"
 
 namespace psattn {
 

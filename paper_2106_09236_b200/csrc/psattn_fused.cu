@@ -27,6 +27,7 @@ struct FusedArgs {
     uint32_t off_persist;                // M~, selection, flags: live through all phases
     int pos_t, pos_h, pos_b;             // TMA coordinate slots (same for the three maps)
     int own_v;                           // fill with the query's own value row instead of mean(V)
+    int by_length;                       // CTAs take the sequences in descending order of length
 };
 
 struct FusedPersist {                    // at smem + off_persist + 4 * T (after the M~ array)
@@ -44,7 +45,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     const __grid_constant__ CUtensorMap tmV) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int unit = blockIdx.x, b = unit / g.H, h = unit % g.H;
     float *M_s = reinterpret_cast<float *>(smem + a.off_persist);
     unsigned char *chosen = reinterpret_cast<unsigned char *>(M_s + g.T);
     FusedPersist &P = *reinterpret_cast<FusedPersist *>(smem + a.off_persist + ((5 * (size_t)g.T + 127) / 128) * 128);
@@ -60,6 +60,27 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (warp == 0) tmem_alloc(&P.tmem_slot, kA64TmemCols);
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Which unit this CTA works on.  With ragged lengths the CTAs take the sequences longest first
+    // (CTA x gets the sequence of rank x / H in descending length, ties by position): when there are
+    // more units than SMs the long ones start in the first wave and the short ones fill the tail.
+    int b = blockIdx.x / g.H;
+    const int h = blockIdx.x % g.H;
+    if (a.by_length) {
+        __shared__ int b_ranked;
+        const int rank = b;
+        for (int c = tid; c < g.B; c += kFusedThreads) {
+            const int lc = min(max(g.lengths[c], 0), g.T);
+            int before = 0;
+            for (int o = 0; o < g.B; ++o) {
+                const int lo = min(max(g.lengths[o], 0), g.T);
+                before += (lo > lc) || (lo == lc && o < c);
+            }
+            if (before == rank) b_ranked = c;
+        }
+        __syncthreads();
+        b = b_ranked;
+    }
+    const int unit = b * g.H + h;
     const int L = seq_len(g, b);
     const int U = min(g.U_tab[L], g.idx_cols);
     const int u = min(min(g.u_tab[L], g.u_max), L);
@@ -173,6 +194,8 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
         if (p0[x] != p1[x] || p1[x] != p2[x]) return cudaErrorNotSupported;
     a.pos_t = p0[0]; a.pos_h = p0[1]; a.pos_b = p0[2];
     a.own_v = own_v;
+    // the ranking costs B comparisons per sequence in every CTA: only where a second wave exists and B is small
+    a.by_length = g.lengths != nullptr && g.B * g.H > kSmCount && g.B <= 256;
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
         cudaError_t e = cudaFuncSetAttribute(k_forward_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -8,6 +8,7 @@ constexpr int kColsumRows = 256;      // rows of V per column-sum partial
 constexpr int kFillRows = 128;        // rows of O per fill block
 constexpr int kSelectThreads = 1024;
 constexpr int kSelectSmemKeys = 8192; // keys kept in shared memory by the select kernel (32 KB)
+constexpr int kSmCount = 148;         // SMs of a B200
 constexpr int kSplitKeys = 1024;      // keys per split of the SIMT attention kernel
 
 // Every kernel launch of the library is counted (process-wide).

@@ -10,7 +10,8 @@
 //   warpgroup        masked online softmax of (row, tile) per thread; P_a, P_b (bf16) -> shared memory
 //   control thread   O_a = P_a V_a, O_b = P_b V_b -> TMEM
 //   warpgroup        acc = acc * alpha + O
-// The control thread is a small polling scheduler so that neither warpgroup waits for the other.
+// Each warpgroup has its own control thread (lane 0 of warps ctrl_warp and ctrl_warp + 1), so neither
+// waits for the other; the scores of the next pair are issued as soon as the warpgroup has read the current ones.
 // At the end the (m, l, acc) states of the two tiles of a pair and of the two warpgroups are merged.
 // Every wait is bounded; on expiry the routine sets the status bit and unwinds.
 #pragma once
@@ -34,7 +35,7 @@ struct Attend64Job {
     const int *rows;             // listed positions (global or shared), or null = identity
     int n_rows;                  // <= 64
     int pos_t, pos_h, pos_b;     // TMA coordinate slots
-    int ctrl_warp, wg_warp0;     // warp of the control thread; first warp of warpgroup 0 (multiple of 4)
+    int ctrl_warp, wg_warp0;     // warps ctrl_warp, ctrl_warp + 1: control threads; first warp of warpgroup 0 (multiple of 4)
     int started;                 // attend64_start was already run for this job
     int sum_row;                 // slot (>= n_rows, < 64) kept active although it lists no query: its zero
                                  // query row gets weight 1 on every key, so it returns the column sums of V
@@ -180,64 +181,57 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
 #pragma unroll
     for (int c = 0; c < kD; ++c) acc[c] = 0.f;
 
-    if (warp == j.ctrl_warp) {
-        if (lane == 0 && n_pairs > 0) {
-            // ------------------------------ control thread ------------------------------------------
+    if (warp >= j.ctrl_warp && warp < j.ctrl_warp + 2) {
+        const int wg = warp - j.ctrl_warp;
+        if (lane == 0 && wg < n_pairs) {
+            // ---------------- control thread of warpgroup wg: a straight-line program per pair -------------
             constexpr uint32_t kIdescS = umma_idesc_bf16(64, 128, 0);       // B = K tile, K-major
             constexpr uint32_t kIdescO = umma_idesc_bf16(64, kD, 1);        // B = V tile, MN-major
-            int q_of[2] = {0, 1}, stage[2] = {0, 0}, k_pref[2] = {0, 0};
-            const unsigned long long t0 = global_ns();
-            unsigned polls = 0;
-            while ((q_of[0] < n_pairs || q_of[1] < n_pairs) && !*abort_flag) {
-                for (int wg = 0; wg < 2; ++wg) {
-                    const int q = q_of[wg];
-                    if (q >= n_pairs) continue;
-                    const uint32_t ph = (uint32_t)((q >> 1) & 1);
-                    const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
-                    const uint32_t wg_smem = smem_u32(smem + kA64OffWg + wg * kA64WgBytes);
-                    const uint32_t t_s = tmem_base + wg * 192, t_o = t_s + 128;
-                    if (stage[wg] == 0) {
-                        if (mbar_test(&kfull[wg], ph)) {
-                            tc_fence_after();
-                            const uint32_t qa = smem_u32(smem + kA64OffQ);
-                            for (int s = 0; s <= two; ++s)
+            const uint32_t wg_smem = smem_u32(smem + kA64OffWg + wg * kA64WgBytes);
+            const uint32_t qa = smem_u32(smem + kA64OffQ);
+            const uint32_t t_s = tmem_base + wg * 192, t_o = t_s + 128;
+            auto issue_s = [&](int q) {                        // S_a = Q K_a^T, S_b = Q K_b^T
+                const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
+                for (int s = 0; s <= two; ++s)
 #pragma unroll
-                                for (int k = 0; k < kD / 16; ++k)
-                                    umma_bf16(t_s + ((uint32_t)(16 * s) << 16), umma_desc_sw128(qa + k * 32, 16, 1024),
-                                              umma_desc_sw128(wg_smem + s * kA64Tile + k * 32, 16, 1024), kIdescS, k > 0);
-                            umma_commit(&sfull[wg]);
-                            stage[wg] = 1;
-                        }
-                    } else if (stage[wg] == 1) {
-                        if (!k_pref[wg] && q + 2 < n_pairs && mbar_test(&sfull[wg], ph)) {
-                            load_pair(wg, q + 2, false);        // the K buffers are free once S is done
-                            k_pref[wg] = 1;
-                        }
-                        if (mbar_test(&pready[wg], ph) && mbar_test(&vfull[wg], ph)) {
-                            tc_fence_after();
-                            for (int s = 0; s <= two; ++s)
+                    for (int k = 0; k < kD / 16; ++k)
+                        umma_bf16(t_s + ((uint32_t)(16 * s) << 16), umma_desc_sw128(qa + k * 32, 16, 1024),
+                                  umma_desc_sw128(wg_smem + s * kA64Tile + k * 32, 16, 1024), kIdescS, k > 0);
+                umma_commit(&sfull[wg]);
+            };
+            auto give_up = [&]() { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); };
+            bool alive = !*abort_flag;
+            if (alive && !mbar_wait(&kfull[wg], 0)) { give_up(); alive = false; }
+            if (alive) { tc_fence_after(); issue_s(wg); }
+            int cnt = 0;
+            for (int q = wg; alive && q < n_pairs; q += 2, ++cnt) {
+                const uint32_t ph = (uint32_t)(cnt & 1);
+                const bool more = q + 2 < n_pairs;
+                const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
+                // the K buffers are free once S is done: bring in the next pair's keys
+                if (!mbar_wait(&sfull[wg], ph)) { give_up(); break; }
+                if (more) load_pair(wg, q + 2, false);
+                // O_a = P_a V_a, O_b = P_b V_b once the warpgroup has written P
+                if (!mbar_wait(&pready[wg], ph) || !mbar_wait(&vfull[wg], ph)) { give_up(); break; }
+                tc_fence_after();
+                for (int s = 0; s <= two; ++s)
 #pragma unroll
-                                for (int k = 0; k < 8; ++k)
-                                    umma_bf16(t_o + ((uint32_t)(16 * s) << 16),
-                                              umma_desc_sw128(wg_smem + (4 + s) * kA64Tile + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024),
-                                              umma_desc_sw128(wg_smem + (2 + s) * kA64Tile + k * 2048, 16, 1024), kIdescO, k > 0);
-                            umma_commit(&ofull[wg]);
-                            stage[wg] = 2;
-                        }
-                    } else {
-                        if (mbar_test(&ofull[wg], ph)) {
-                            if (q + 2 < n_pairs) {
-                                if (!k_pref[wg]) load_pair(wg, q + 2, false);
-                                load_pair(wg, q + 2, true);
-                            }
-                            q_of[wg] = q + 2; k_pref[wg] = 0; stage[wg] = 0;
-                        }
-                    }
+                    for (int k = 0; k < 8; ++k)
+                        umma_bf16(t_o + ((uint32_t)(16 * s) << 16),
+                                  umma_desc_sw128(wg_smem + (4 + s) * kA64Tile + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024),
+                                  umma_desc_sw128(wg_smem + (2 + s) * kA64Tile + k * 2048, 16, 1024), kIdescO, k > 0);
+                umma_commit(&ofull[wg]);
+                // the warpgroup has read S (it signalled P): the next pair's scores can be computed while it
+                // adds O of this pair to its accumulators
+                if (more) {
+                    if (!mbar_wait(&kfull[wg], ph ^ 1u)) { give_up(); break; }
+                    tc_fence_after();
+                    issue_s(q + 2);
                 }
-                if ((++polls & 255u) == 0u && global_ns() - t0 > 2 * kWaitNs) {
-                    *abort_flag = 1u;
-                    atomicOr(g.status, kStatusWaitExpired);
-                }
+                // the V buffers are free once O is done
+                if (!mbar_wait(&ofull[wg], ph)) { give_up(); break; }
+                if (more) load_pair(wg, q + 2, true);
+                if (*abort_flag) break;
             }
         }
     } else if (warp >= j.wg_warp0 && warp < j.wg_warp0 + 8) {

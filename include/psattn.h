@@ -33,7 +33,8 @@
  *   - sample_idx: device int32, row (b, i) (or (b, h, i) with idx_per_head) holds the sampled
  *     key positions of query i in its first U_b entries; row stride idx_cols elements.  Entries
  *     must lie in [0, lengths[b]); others are clamped into range and status bit 0 is set.
- *     A key that occurs twice counts twice in the mean of Eq. 11.
+ *     A key that occurs twice counts twice in the mean of Eq. 11.  With idx_shared the array has
+ *     one row per sequence (or per unit) instead of one per query.
  *   - sel_idx: device int32 [B][H][u_max], the selected query positions of each unit in
  *     ascending order, padded with -1.  Equal M~ values are ordered by position (lower first).
  *   - workspace: device scratch of at least psattn_workspace_bytes() bytes, 256-byte aligned.
@@ -84,7 +85,9 @@ typedef struct psattn_desc {
     int32_t idx_per_head;               /* 0: sample_idx is [B][T_max][idx_cols], shared by the heads;
                                            1: [B][H][T_max][idx_cols] */
     int32_t path;                       /* PSATTN_PATH_*: kernel schedule; AUTO picks per shape */
-    int32_t reserved;
+    int32_t idx_shared;                 /* 1: one sample per sequence, used by all its queries (the other
+                                           reading of "a random sampling key matrix", Sec. 3.2): sample_idx
+                                           is [B][idx_cols] (or [B][H][idx_cols] with idx_per_head) */
     double c;                           /* sampling factor of n(c, len) */
     int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* b, h, t strides in elements; all 0 = dense */
 } psattn_desc_t;

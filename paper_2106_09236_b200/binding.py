@@ -31,7 +31,7 @@ class psattn_desc_t(ctypes.Structure):
         ("d_head", ctypes.c_int32), ("dtype", ctypes.c_int32), ("fill_mode", ctypes.c_int32),
         ("u_override", ctypes.c_int32), ("U_override", ctypes.c_int32),
         ("idx_cols", ctypes.c_int32), ("idx_per_head", ctypes.c_int32),
-        ("path", ctypes.c_int32), ("reserved", ctypes.c_int32), ("c", ctypes.c_double),
+        ("path", ctypes.c_int32), ("idx_shared", ctypes.c_int32), ("c", ctypes.c_double),
         ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
         ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3),
     ]
@@ -131,7 +131,7 @@ class Plan:
 
     def __init__(self, B, H, T_max, dtype=torch.bfloat16, c=5.0, idx_cols=None, d_head=64,
                  fill_mode=PSATTN_FILL_MEAN_V, u_override=0, U_override=0, idx_per_head=False,
-                 path=PSATTN_PATH_AUTO, strides=None):
+                 path=PSATTN_PATH_AUTO, strides=None, idx_shared=False):
         lib = load()
         self.lib = lib
         d = psattn_desc_t()
@@ -142,6 +142,7 @@ class Plan:
             idx_cols = U_override if U_override > 0 else max(
                 [psattn_count(c, L) for L in range(1, T_max + 1)] + [1])
         d.idx_cols, d.idx_per_head, d.path, d.c = idx_cols, int(idx_per_head), path, c
+        d.idx_shared = int(idx_shared)
         if strides is not None:
             for name in ("q", "k", "v", "o"):
                 if name in strides:

@@ -93,6 +93,7 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     if (d.fill_mode != PSATTN_FILL_MEAN_V && d.fill_mode != PSATTN_FILL_OWN_V) return PSATTN_ERR_BAD_DESC;
     if (d.path < PSATTN_PATH_AUTO || d.path > PSATTN_PATH_FUSED) return PSATTN_ERR_BAD_DESC;
     if (d.u_override < 0 || d.U_override < 0 || d.idx_cols < 1) return PSATTN_ERR_BAD_DESC;
+    if (d.idx_shared != 0 && d.idx_shared != 1) return PSATTN_ERR_BAD_DESC;
     if (!(d.c > 0.0) || !std::isfinite(d.c)) return PSATTN_ERR_BAD_DESC;
     if (d.d_head != kD) return PSATTN_ERR_UNSUPPORTED;
     int rc;
@@ -200,7 +201,7 @@ static Geom make_geom(const psattn_plan_t *p, const int32_t *lengths, void *ws) 
     Geom g;
     const psattn_desc_t &d = p->desc;
     g.B = plan_b(p); g.H = d.H; g.T = d.T_max;
-    g.idx_cols = d.idx_cols; g.idx_per_head = d.idx_per_head;
+    g.idx_cols = d.idx_cols; g.idx_per_head = d.idx_per_head; g.idx_shared = d.idx_shared;
     g.u_max = p->u_max;
     for (int k = 0; k < 3; ++k) {
         g.qs[k] = d.q_stride[k]; g.ks[k] = d.k_stride[k];
@@ -226,6 +227,16 @@ static T *ws_at(void *ws, size_t off) { return reinterpret_cast<T *>(static_cast
 static int run_measure(psattn_plan_t *plan, const Geom &g, const void *Q, const void *K,
                        const int *sample_idx, float *M, cudaStream_t st) {
     const psattn_desc_t &d = plan->desc;
+    if (d.idx_shared) {
+        // one sample per sequence: the scores of a tile of queries are one dense product on tcgen05
+        if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
+            cudaError_t e = launch_measure_shared(g, plan->U_max, Q, K, sample_idx, M, st);
+            if (e == cudaSuccess) return PSATTN_OK;
+            if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+        }
+        PSATTN_CU(launch_measure(d.dtype, g, Q, K, sample_idx, M, st));
+        return PSATTN_OK;
+    }
     if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
         cudaError_t e = launch_measure_mma(g, plan->U_max, Q, K, sample_idx, M, st);
         if (e == cudaSuccess) return PSATTN_OK;
@@ -330,7 +341,7 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
-    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && !d.idx_shared) {
         cudaError_t e = launch_forward_fused(g, plan->U_max, d.fill_mode == PSATTN_FILL_OWN_V, Q, K, V, sample_idx, O,
                                              sel_idx, M_out, st);
         if (e == cudaSuccess) return PSATTN_OK;
@@ -459,7 +470,7 @@ extern "C" int psattn_plan_enable_host_io(psattn_plan_t *plan) {
     const psattn_desc_t &d = plan->desc;
     const size_t es = d.dtype == PSATTN_BF16 ? 2 : 4;
     const size_t n = (size_t)d.B * d.H * d.T_max * kD * es;
-    const size_t nidx = (size_t)d.B * (d.idx_per_head ? d.H : 1) * d.T_max * d.idx_cols * sizeof(int);
+    const size_t nidx = (size_t)d.B * (d.idx_per_head ? d.H : 1) * (d.idx_shared ? 1 : d.T_max) * d.idx_cols * sizeof(int);
     void **bufs[] = {&plan->h_Q, &plan->h_K, &plan->h_V, &plan->h_O, &plan->h_ws,
                      (void **)&plan->h_len, (void **)&plan->h_idx, (void **)&plan->h_sel};
     const size_t sizes[] = {n, n, n, n, plan->ws_bytes, (size_t)d.B * sizeof(int) + 16, nidx + 16,
@@ -491,7 +502,7 @@ extern "C" int psattn_forward_host(psattn_plan_t *plan, const void *Q, const voi
     // computed on `stream`, the results of chunk k - 1 travel back on a second stream (PCIe is full
     // duplex).  All chunks share the one workspace; they are ordered by `stream`.
     const size_t per_b = (size_t)d.H * d.T_max * kD * es;
-    const size_t idx_b = (size_t)(d.idx_per_head ? d.H : 1) * d.T_max * d.idx_cols * sizeof(int);
+    const size_t idx_b = (size_t)(d.idx_per_head ? d.H : 1) * (d.idx_shared ? 1 : d.T_max) * d.idx_cols * sizeof(int);
     const size_t sel_b = (size_t)d.H * plan->u_max * sizeof(int);
     if (lengths) PSATTN_CU(cudaMemcpyAsync(plan->h_len, lengths, (size_t)d.B * sizeof(int), cudaMemcpyHostToDevice, st));
     // the staging buffers are dense: run with dense strides whatever the descriptor says

@@ -18,6 +18,7 @@ constexpr unsigned kStatusWaitExpired = 4u;
 struct Geom {
     int B, H, T;                          // T = T_max
     int idx_cols, idx_per_head;
+    int idx_shared;                       // one sample row per sequence (or unit) instead of one per query
     int u_max;
     long long qs[3], ks[3], vs[3], os[3]; // element strides of the b, h, t axes
     const int *lengths;                   // device, may be null

@@ -30,6 +30,9 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
 // through shared-memory rings); cudaErrorNotSupported when U_max > 64.
 cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
                                   cudaStream_t st);
+// One sample per sequence (Geom::idx_shared): the scores of 128 queries are one tcgen05 product.
+cudaError_t launch_measure_shared(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
+                                  cudaStream_t st);
 cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, int n_chunks,
                           cudaStream_t st);
 cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,

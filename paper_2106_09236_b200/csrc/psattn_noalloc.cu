@@ -76,7 +76,7 @@ extern "C" int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, floa
 
     Geom g;
     g.B = B; g.H = H; g.T = T_max;
-    g.idx_cols = 0; g.idx_per_head = 0; g.u_max = 0;
+    g.idx_cols = 0; g.idx_per_head = 0; g.idx_shared = 0; g.u_max = 0;
     const long long dense[3] = {(long long)H * T_max * kD, (long long)T_max * kD, kD};
     for (int k = 0; k < 3; ++k) { g.qs[k] = g.ks[k] = g.vs[k] = g.os[k] = dense[k]; }
     g.lengths = lengths;

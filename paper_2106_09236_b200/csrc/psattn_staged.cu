@@ -34,7 +34,8 @@ __global__ void __launch_bounds__(256) k_measure(Geom g, const DT *__restrict__ 
     float q[8];
     load8(Q + unit_off(g.qs, b, h) + (long long)i * g.qs[2], sub, q);
     const DT *Ku = K + unit_off(g.ks, b, h);
-    const int *row = sidx + ((g.idx_per_head ? (long long)unit : (long long)b) * g.T + i) * g.idx_cols;
+    const int *row = sidx + (g.idx_shared ? (g.idx_per_head ? (long long)unit : (long long)b)
+                                          : (g.idx_per_head ? (long long)unit : (long long)b) * g.T + i) * g.idx_cols;
 
     MeasureState st = measure_init();
     for (int base = 0; base < U; base += 32) {

@@ -161,9 +161,10 @@ def test_paper_literal_variant_at_scale(dtype, T, r_sparse):
     parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c, u_override=u, fill="own_v")
 
 
+@pytest.mark.parametrize("T", [80, 1300])           # keys resident in shared memory / streamed from L2
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
-def test_out_of_range_inputs_set_status_bits_without_faulting(path):
-    B, H, T, c = 2, 1, 80, 5.0
+def test_out_of_range_inputs_set_status_bits_without_faulting(path, T):
+    B, H, c = 2, 1, 5.0
     n = orc.count(c, T)
     inp = _synth(B, H, T, 47, n, "bf16")
     bad = {k: v.copy() for k, v in inp.items()}
@@ -243,6 +244,48 @@ def test_measure_per_head_samples():
                             None, torch.from_numpy(idx).cuda())
     torch.cuda.synchronize()
     parity.check_measure(M.cpu().numpy(), orc.measure(inp["Q"], inp["K"], idx, None, c=c))
+    plan.close()
+
+
+# ---- one sample per sequence (the other reading of Sec. 3.2's sampled key matrix) -----------
+
+def _shared_sample(inp):
+    """The compact [B][U] sample (query 0's draw of each sequence) and the per-query array the
+    oracle reads, every query row holding that same sample."""
+    B, H, T, _ = inp["Q"].shape
+    compact = np.ascontiguousarray(inp["sample_idx"][:, 0, :])
+    expanded = np.ascontiguousarray(np.broadcast_to(compact[:, None, :], (B, T, compact.shape[-1])))
+    return compact, expanded
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("dtype,T", [("bf16", 300), ("fp32", 300), ("bf16", 1500)])
+def test_shared_sample_forward(dtype, T, path):
+    B, H, c = 3, 2, 5.0
+    lengths = [T, max(1, T // 3), T - 1]
+    n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+    inp = _synth(B, H, T, 700 + T, n_cols, dtype, lengths)
+    compact, expanded = _shared_sample(inp)
+    O, sel, M, status = _run_forward(dict(inp, sample_idx=compact), dtype, c, path, idx_shared=True)
+    assert status == 0
+    parity.check_forward(O, sel, M, dict(inp, sample_idx=expanded), inp["lengths"], dtype, c)
+
+
+def test_shared_sample_measure_large_and_per_head():
+    w = wl.WORKLOADS["large_bf16"]
+    n = orc.count(w.c, w.T)
+    inp = wl.make_inputs(w, n, B=2)
+    B, H, T = 2, w.H, w.T
+    rng = np.random.default_rng(77)
+    compact = rng.integers(0, T, size=(B, H, n)).astype(np.int32)
+    compact[0, 1, 3] = compact[0, 1, 2]                  # a key drawn twice counts twice
+    expanded = np.ascontiguousarray(np.broadcast_to(compact[:, :, None, :], (B, H, T, n)))
+    plan = ps.Plan(B, H, T, dtype=torch.bfloat16, c=w.c, idx_cols=n, idx_per_head=True, idx_shared=True)
+    dev, _ = _dev(inp, "bf16")
+    M = plan.psattn_measure(dev["Q"], dev["K"], None, torch.from_numpy(compact).cuda())
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() == 0
+    parity.check_measure(M.cpu().numpy(), orc.measure(inp["Q"], inp["K"], expanded, None, c=w.c))
     plan.close()
 
 

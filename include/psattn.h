@@ -136,6 +136,13 @@ int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K, const int3
                    const int32_t *sample_idx, float *M_out, void *workspace,
                    size_t workspace_bytes, void *stream);
 
+/* The exact sparsity measure that Eq. 11 approximates (Eq. 10): M_out[b][h][i] =
+ * ln sum_j exp(s_ij) - (1/len) sum_j s_ij over ALL valid keys j < lengths[b]; fp32 [B][H][T_max],
+ * zero at padded positions.  A dense pass over the score matrix (cost of dense attention's first
+ * half); no sample is involved.  All pointers device. */
+int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const void *K, const int32_t *lengths,
+                         float *M_out, void *workspace, size_t workspace_bytes, void *stream);
+
 /* Step (c) only (Sec. 3.2): top-u positions of M (fp32 [B][H][T_max]) among i < lengths[b]. */
 int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
                   int32_t *sel_idx, void *workspace, size_t workspace_bytes, void *stream);

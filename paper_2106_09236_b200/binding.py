@@ -19,7 +19,7 @@ PSATTN_PATH_AUTO, PSATTN_PATH_STAGED, PSATTN_PATH_FUSED = 0, 1, 2
 EXPORTS = [
     "psattn_version", "psattn_launch_count", "psattn_status_string", "psattn_last_cuda_error", "psattn_count",
     "psattn_plan_create", "psattn_plan_destroy", "psattn_plan_limits", "psattn_workspace_bytes",
-    "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_select",
+    "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_exact_measure", "psattn_select",
     "psattn_mean_v", "psattn_attend_rows", "psattn_dense_forward", "psattn_read_status",
     "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc",
 ]
@@ -73,6 +73,7 @@ def load(build_if_missing: bool = True):
     lib.psattn_forward.argtypes = [vp] * 10 + [sz, vp]
     lib.psattn_forward_with_selection.argtypes = [vp] * 8 + [sz, vp]
     lib.psattn_measure.argtypes = [vp] * 7 + [sz, vp]
+    lib.psattn_exact_measure.argtypes = [vp] * 6 + [sz, vp]
     lib.psattn_select.argtypes = [vp] * 5 + [sz, vp]
     lib.psattn_mean_v.argtypes = [vp] * 5 + [sz, vp]
     lib.psattn_attend_rows.argtypes = [vp] * 6 + [i32, vp, vp, sz, vp]
@@ -202,6 +203,14 @@ class Plan:
         ws, n = self._ws()
         _check(self.lib.psattn_measure(self.handle, _ptr(Q), _ptr(K), _ptr(lengths),
                                        _ptr(sample_idx), _ptr(M_out), ws, n, _stream()), self.handle)
+        return M_out
+
+    def psattn_exact_measure(self, Q, K, lengths, M_out=None):
+        if M_out is None:
+            M_out = torch.empty((self.B, self.H, self.T_max), dtype=torch.float32, device=Q.device)
+        ws, n = self._ws()
+        _check(self.lib.psattn_exact_measure(self.handle, _ptr(Q), _ptr(K), _ptr(lengths), _ptr(M_out),
+                                             ws, n, _stream()), self.handle)
         return M_out
 
     def psattn_select(self, M, lengths, sel_idx=None):

@@ -393,6 +393,20 @@ extern "C" int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K,
     return run_measure(plan, g, Q, K, sample_idx, M_out, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const void *K, const int32_t *lengths,
+                                    float *M_out, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!plan || !Q || !K || !M_out) return PSATTN_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    Geom g = make_geom(plan, lengths, workspace);
+    const psattn_desc_t &d = plan->desc;
+    // PSATTN_PATH_STAGED keeps the arithmetic off the tensor cores (one warp per query)
+    const int dtype = d.dtype == PSATTN_BF16 && d.path == PSATTN_PATH_STAGED ? 2 : d.dtype;
+    PSATTN_CU(launch_exact_measure(dtype, g, Q, K, M_out, static_cast<cudaStream_t>(stream)));
+    return PSATTN_OK;
+}
+
 extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
                              int32_t *sel_idx, void *workspace, size_t workspace_bytes,
                              void *stream) {

@@ -35,7 +35,7 @@ struct AttendTcArgs {
     int pos_t, pos_h, pos_b;    // which TMA coordinate (1..3) carries t, h, b
 };
 
-__global__ void __launch_bounds__(128, 1) k_attend_tc(Geom g, AttendTcArgs a,
+__global__ void __launch_bounds__(128, 2) k_attend_tc(Geom g, AttendTcArgs a,
                                                       const __nv_bfloat16 *__restrict__ Q,
                                                       const __grid_constant__ CUtensorMap tmK,
                                                       const __grid_constant__ CUtensorMap tmV) {
@@ -331,6 +331,10 @@ cudaError_t launch_attend_tc(const Geom &g, const void *Q, const void *K, const 
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttendSmem);
+        // two CTAs fit an SM (2 x 113 KB of shared memory, 2 x 256 TMEM columns) and hide each other's waits
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }

@@ -30,6 +30,8 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
 // through shared-memory rings); cudaErrorNotSupported when U_max > 64.
 cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
                                   cudaStream_t st);
+// Eq. 10 over all valid keys (dense pass): tcgen05 for bf16 (dtype 0), one warp per query otherwise.
+cudaError_t launch_exact_measure(int dtype, const Geom &g, const void *Q, const void *K, float *M, cudaStream_t st);
 // One sample per sequence (Geom::idx_shared): the scores of 128 queries are one tcgen05 product.
 cudaError_t launch_measure_shared(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,
                                   cudaStream_t st);

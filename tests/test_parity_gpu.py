@@ -289,6 +289,26 @@ def test_shared_sample_measure_large_and_per_head():
     plan.close()
 
 
+# ---- the exact measure of Eq. 10 (dense pass) ------------------------------------------------
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("dtype,T", [("bf16", 300), ("bf16", 1100), ("fp32", 150)])
+def test_exact_measure_entry_point(dtype, T, path):
+    """ln sum exp(s) - mean(s) over all valid keys against the oracle's fp64 evaluation of Eq. 10
+    (tensor-core form for bf16 on the automatic path, one warp per query otherwise)."""
+    B, H, c = 2, 3, 5.0
+    lengths = [T, max(1, T - 129)]
+    inp = _synth(B, H, T, 900 + T, orc.count(c, T), dtype, lengths)
+    dev, tdt = _dev(inp, dtype)
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, path=path)
+    M = plan.psattn_exact_measure(dev["Q"], dev["K"], dev["lengths"])
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() == 0
+    plan.close()
+    ref = orc.exact_measure(inp["Q"], inp["K"], inp["lengths"])
+    parity.check_measure(M.cpu().numpy(), ref, inp["lengths"])
+
+
 def test_select_entry_point_is_exact_including_ties():
     B, H, T, c = 3, 2, 700, 5.0
     rng = np.random.default_rng(50)

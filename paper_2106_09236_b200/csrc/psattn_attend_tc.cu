@@ -115,61 +115,71 @@ __global__ void __launch_bounds__(128, 2) k_attend_tc(Geom g, AttendTcArgs a,
     for (int c = 0; c < kD; ++c) acc[c] = 0.f;
     const bool warp_has_rows = (row_tile * kTileRows + warp * 32) < a.n_rows;
 
+    // thread 0: S = Q K^T of key tile t once the tile has landed (the S accumulator must be free)
+    auto issue_s = [&](int t) {
+        const int s = t & 1;
+        if (!mbar_wait(&full_k[s], (uint32_t)((t >> 1) & 1))) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); return; }
+        tc_fence_after();
+        const uint32_t qa = smem_u32(smem + kOffQ), ka = smem_u32(smem + kOffK + s * kTileBytes);
+#pragma unroll
+        for (int k = 0; k < kD / 16; ++k)
+            umma_bf16(tmem_base, umma_desc_sw128(qa + k * 32, 16, 1024), umma_desc_sw128(ka + k * 32, 16, 1024),
+                      kIdescS, k > 0);
+        umma_commit(mma_s);
+    };
+    if (tid == 0 && n_tiles > 0) issue_s(0);
+
     for (int t = 0; t < n_tiles; ++t) {
         const int s = t & 1;
         const uint32_t ph_load = (uint32_t)((t >> 1) & 1), ph_mma = (uint32_t)(t & 1);
-        // ---- S = Q K^T -----------------------------------------------------------------
-        if (tid == 0 && !*abort_flag) {
-            if (!mbar_wait(&full_k[s], ph_load)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); }
-            else {
-                tc_fence_after();
-                const uint32_t qa = smem_u32(smem + kOffQ), ka = smem_u32(smem + kOffK + s * kTileBytes);
-#pragma unroll
-                for (int k = 0; k < kD / 16; ++k)
-                    umma_bf16(tmem_base, umma_desc_sw128(qa + k * 32, 16, 1024),
-                              umma_desc_sw128(ka + k * 32, 16, 1024), kIdescS, k > 0);
-                umma_commit(mma_s);
-            }
-        }
+        __syncwarp();
         if (!*abort_flag && !mbar_wait(mma_s, ph_mma)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); }
         tc_fence_after();
         // ---- masked online softmax of this thread's row; P -> shared memory -------------------
+        // two passes over the 128 scores in TMEM, 64 at a time with both loads of a half in flight
         const int valid = min(kTileKeys, hi - (lo + t * kTileKeys));     // keys of this tile that exist
         float alpha = 1.f;
         __syncwarp();
         if (warp_has_rows && !*abort_flag) {
+            uint32_t sv[2][32];
             float mx = -INFINITY;
 #pragma unroll
-            for (int cb = 0; cb < 4; ++cb) {
-                float v[32];
-                tmem_ld32(lane_base + cb * 32, v);
+            for (int hf = 0; hf < 2; ++hf) {
+                tmem_ld32_issue(lane_base + hf * 64, sv[0]);
+                tmem_ld32_issue(lane_base + hf * 64 + 32, sv[1]);
+                tmem_ld_wait();
+                tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) if (cb * 32 + j < valid) mx = fmaxf(mx, v[j]);
+                for (int x = 0; x < 64; ++x)
+                    if (hf * 64 + x < valid) mx = fmaxf(mx, __uint_as_float(sv[x >> 5][x & 31]));
             }
             const float m_new = fmaxf(m_run, mx * kScaleLog2);
-            alpha = exp2f(m_run - m_new);                       // 0 on the first tile
+            alpha = fast_exp2(m_run - m_new);                   // 0 on the first tile
             float lsum = 0.f;
 #pragma unroll
-            for (int cb = 0; cb < 4; ++cb) {
-                float v[32];
-                tmem_ld32(lane_base + cb * 32, v);
-                uint32_t packed[16];
+            for (int hf = 0; hf < 2; ++hf) {
+                tmem_ld32_issue(lane_base + hf * 64, sv[0]);
+                tmem_ld32_issue(lane_base + hf * 64 + 32, sv[1]);
+                tmem_ld_wait();
+                tmem_ld_fence32(sv[0]); tmem_ld_fence32(sv[1]);
+                uint8_t *prow = smem + kOffP + hf * kTileBytes + tid * 128;    // panel hf: keys 64 * hf ..
 #pragma unroll
-                for (int j = 0; j < 32; j += 2) {
-                    float p0 = (cb * 32 + j < valid) ? exp2f(fmaf(v[j], kScaleLog2, -m_new)) : 0.f;
-                    float p1 = (cb * 32 + j + 1 < valid) ? exp2f(fmaf(v[j + 1], kScaleLog2, -m_new)) : 0.f;
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    // the weights that multiply V are the rounded ones: sum those for the denominator
-                    lsum += __low2float(pk) + __high2float(pk);
-                    packed[j >> 1] = *reinterpret_cast<uint32_t *>(&pk);
-                }
-                // 32 keys = 64 bytes = 4 chunks of 16 bytes; panel = cb / 2, chunk = (cb % 2) * 4 + q
-                uint8_t *prow = smem + kOffP + (cb >> 1) * kTileBytes + tid * 128;
+                for (int ch = 0; ch < 8; ++ch) {                // 8 keys = one 16-byte chunk
+                    uint32_t packed[4];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int chunk = (cb & 1) * 4 + q4;
-                    *reinterpret_cast<uint4 *>(prow + ((chunk ^ (tid & 7)) << 4)) =
-                        make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
+                    for (int x = 0; x < 8; x += 2) {
+                        const int col = ch * 8 + x;
+                        const float s0 = __uint_as_float(sv[col >> 5][col & 31]);
+                        const float s1 = __uint_as_float(sv[(col + 1) >> 5][(col + 1) & 31]);
+                        const float p0 = (hf * 64 + col < valid) ? fast_exp2(fmaf(s0, kScaleLog2, -m_new)) : 0.f;
+                        const float p1 = (hf * 64 + col + 1 < valid) ? fast_exp2(fmaf(s1, kScaleLog2, -m_new)) : 0.f;
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                        // the weights that multiply V are the rounded ones: sum those for the denominator
+                        lsum += __low2float(pk) + __high2float(pk);
+                        packed[x >> 1] = *reinterpret_cast<uint32_t *>(&pk);
+                    }
+                    *reinterpret_cast<uint4 *>(prow + ((ch ^ (tid & 7)) << 4)) =
+                        make_uint4(packed[0], packed[1], packed[2], packed[3]);
                 }
             }
             l_run = l_run * alpha + lsum;
@@ -186,8 +196,8 @@ __global__ void __launch_bounds__(128, 2) k_attend_tc(Geom g, AttendTcArgs a,
         }
         fence_proxy_async_smem();
         tc_fence_before();
-        __syncthreads();
-        // ---- O_t = P V --------------------------------------------------------------------
+        __syncthreads();                                        // P is written, everybody has read S
+        // ---- O_t = P V, then S of the next tile while the threads add O_t ---------------------
         if (tid == 0 && !*abort_flag) {
             if (!mbar_wait(&full_v[s], ph_load)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); }
             else {
@@ -199,22 +209,24 @@ __global__ void __launch_bounds__(128, 2) k_attend_tc(Geom g, AttendTcArgs a,
                               umma_desc_sw128(pa + (k >> 2) * kTileBytes + (k & 3) * 32, 16, 1024),
                               umma_desc_sw128(va + k * 2048, 16, 1024), kIdescO, k > 0);
                 umma_commit(mma_o);
+                if (t + 1 < n_tiles) issue_s(t + 1);
             }
         }
+        __syncwarp();
         if (!*abort_flag && !mbar_wait(mma_o, ph_mma)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); }
         tc_fence_after();
         __syncwarp();
         if (warp_has_rows && !*abort_flag) {
+            uint32_t ov[2][32];
+            tmem_ld32_issue(lane_base + 128, ov[0]);
+            tmem_ld32_issue(lane_base + 160, ov[1]);
+            tmem_ld_wait();
+            tmem_ld_fence32(ov[0]); tmem_ld_fence32(ov[1]);
 #pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                float v[32];
-                tmem_ld32(lane_base + 128 + cb * 32, v);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) acc[cb * 32 + j] = fmaf(acc[cb * 32 + j], alpha, v[j]);
-            }
+            for (int x = 0; x < 64; ++x) acc[x] = fmaf(acc[x], alpha, __uint_as_float(ov[x >> 5][x & 31]));
         }
         tc_fence_before();
-        __syncthreads();                                        // stage s, P, S and O_t are free again
+        __syncthreads();                                        // stage s, P and O_t are free again
         if (tid == 0 && !*abort_flag && loads_issued < n_tiles) { issue_loads(loads_issued); ++loads_issued; }
     }
 

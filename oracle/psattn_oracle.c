@@ -8,6 +8,7 @@
  * library never calls it.
  *
  * Every function follows one passage of the paper (arXiv 2106.09236):
+ *   Sec. 3.1  the projections Q = X W_q, K = X W_k, V = X W_v
  *   Eq. 6-8   dense scaled dot-product attention and its per-query form
  *   Eq. 9-10  the KL-motivated sparsity measure  M = LSE - mean
  *   Eq. 11    its sampled approximation          M~ = max - mean over K~
@@ -291,6 +292,37 @@ void psattn_oracle_dense(const float *Q, const float *K, const float *V, int B, 
             if (i < L) psattn_oracle_attend_row(Q, K, V, H, T, d, L, b, h, i, o);
             else for (int t = 0; t < d; ++t) o[t] = 0.0;
         }
+    }
+}
+
+/*
+ * Sec. 3.1: the projections that precede the attention, Q = X W_q, K = X W_k, V = X W_v,
+ * one (d_x x d) matrix per head and per role.
+ *   X   float  [B][T][d_x]
+ *   Wt  float  [3][H*d][d_x]   role r (0 = q, 1 = k, 2 = v), row h*d + e holds column e of
+ *                              head h's matrix: Wt[r][h*d + e][x] = W_r^h[x][e]
+ *   out double [3][B][H][T][d] out[r][b][h][t][e] = sum_x X[b][t][x] * W_r^h[x][e]
+ * Rows at positions >= len_b are zero (the attention never reads them).
+ */
+void psattn_oracle_project_qkv(const float *X, const float *Wt, int B, int T, int dx, int H,
+                               int d, const int *lengths, double *out, int nthreads) {
+    size_t plane = (size_t)B * H * T * d;
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(nthreads > 0 ? nthreads : 1) schedule(static)
+#endif
+    for (long bt = 0; bt < (long)B * T; ++bt) {
+        int b = (int)(bt / T), t = (int)(bt % T);
+        int L = seq_len(lengths, b, T);
+        const float *x = X + (size_t)bt * dx;
+        for (int r = 0; r < 3; ++r)
+            for (int h = 0; h < H; ++h)
+                for (int e = 0; e < d; ++e) {
+                    const float *w = Wt + ((size_t)r * H * d + (size_t)h * d + e) * dx;
+                    double acc = 0.0;
+                    if (t < L)
+                        for (int k = 0; k < dx; ++k) acc += (double)x[k] * (double)w[k];
+                    out[r * plane + (((size_t)b * H + h) * T + t) * d + e] = acc;
+                }
     }
 }
 

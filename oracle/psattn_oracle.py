@@ -189,3 +189,20 @@ def dense(Q, K, V, lengths=None, nthreads=1):
     O = np.zeros((B, H, T, d), dtype=np.float64)
     lib.psattn_oracle_dense(qp, kp, vp, B, H, T, d, lp, O.ctypes.data_as(_f64p), int(nthreads))
     return O
+
+
+def project_qkv(X, Wt, H, lengths=None, nthreads=1):
+    """Sec. 3.1: Q = X W_q, K = X W_k, V = X W_v per head.  X [B, T, d_x]; Wt [3, H*d, d_x] holds the
+    matrices transposed (row h*d + e = column e of head h).  Returns float64 (Q, K, V), each
+    [B, H, T, d], zero at padded positions."""
+    lib = _load()
+    X, xp = _f32(X)
+    Wt, wp = _f32(Wt)
+    B, T, dx = X.shape
+    assert Wt.ndim == 3 and Wt.shape[0] == 3 and Wt.shape[2] == dx and Wt.shape[1] % H == 0
+    d = Wt.shape[1] // H
+    lengths, lp = _i32(lengths)
+    out = np.zeros((3, B, H, T, d), dtype=np.float64)
+    lib.psattn_oracle_project_qkv(xp, wp, B, T, dx, int(H), d, lp, out.ctypes.data_as(_f64p),
+                                  int(nthreads))
+    return out[0], out[1], out[2]

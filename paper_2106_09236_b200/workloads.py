@@ -108,3 +108,30 @@ def make_inputs(w: Workload, n_cols: int, seed: int | None = None, B: int | None
     if w.dtype == "bf16":
         Q, K, V = round_to_bf16(Q), round_to_bf16(K), round_to_bf16(V)
     return {"Q": Q, "K": K, "V": V, "lengths": lengths, "sample_idx": sample_idx, "peaky": peaky}
+
+
+def make_projection_inputs(w: Workload, seed: int | None = None, B: int | None = None, lengths=None,
+                           pad_value: float = 0.0):
+    """Draw the inputs of the projections that precede the attention (Sec. 3.1): the layer input
+    X float32 [B, T, d_x] with d_x = H * d (the model width of Sec. 4.2), i.i.d. N(0, 1), and the
+    three weight matrices stored transposed, Wt float32 [3, H*d, d_x], i.i.d. N(0, 1/d_x) so that
+    projected values have unit variance.  Rounded to bf16 values when w.dtype == "bf16".  Rows of X
+    at padded positions hold `pad_value`.  Draw order: lengths, X, Wt."""
+    rng = np.random.default_rng((w.seed if seed is None else seed) + 7919)
+    nb = w.B if B is None else B
+    dx = w.H * w.d
+    if lengths is not None:
+        lengths = np.asarray(lengths, dtype=np.int32)
+        nb = int(lengths.shape[0])
+    elif w.ragged is not None:
+        lengths = rng.integers(w.ragged[0], w.ragged[1] + 1, size=nb).astype(np.int32)
+    else:
+        lengths = np.full(nb, w.T, dtype=np.int32)
+    X = rng.standard_normal((nb, w.T, dx), dtype=np.float32)
+    Wt = rng.standard_normal((3, w.H * w.d, dx), dtype=np.float32) / np.float32(np.sqrt(dx))
+    for b in range(nb):
+        if int(lengths[b]) < w.T:
+            X[b, int(lengths[b]):] = pad_value
+    if w.dtype == "bf16":
+        X, Wt = round_to_bf16(X), round_to_bf16(Wt)
+    return {"X": X, "Wt": Wt, "lengths": lengths}

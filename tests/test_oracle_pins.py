@@ -369,3 +369,76 @@ def test_peaky_queries_dominate_selection_on_tiny_workload():
     total = int((sel >= 0).sum())
     assert total == w.H * n
     assert hits >= 0.3 * total      # 13 peaky of 128 per head; chance level would be ~10 %
+
+
+# ---- projections (Sec. 3.1: Q = X W_q, K = X W_k, V = X W_v) ----------------------------------
+def _proj_rand(B, T, dx, H, d, seed):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((B, T, dx)).astype(np.float32)
+    Wt = rng.standard_normal((3, H * d, dx)).astype(np.float32)
+    return X, Wt
+
+
+def test_projection_equals_library_matmul():
+    # the definition written with a library routine: per head, X @ W with W = Wt-slice transposed
+    B, T, dx, H, d = 2, 7, 12, 3, 5
+    X, Wt = _proj_rand(B, T, dx, H, d, 11)
+    got = orc.project_qkv(X, Wt, H)
+    for r in range(3):
+        for h in range(H):
+            W = Wt[r, h * d:(h + 1) * d, :].astype(np.float64).T          # (d_x, d)
+            want = X.astype(np.float64) @ W                               # (B, T, d)
+            np.testing.assert_allclose(got[r][:, h], want, rtol=1e-13, atol=1e-13)
+
+
+def test_projection_identity_and_one_hot_cases():
+    # W_q = I, W_k = 2 I, W_v = a cyclic shift of the columns: each head reads its own slice of X
+    B, T, H, d = 1, 4, 2, 3
+    dx = H * d
+    rng = np.random.default_rng(5)
+    X = rng.standard_normal((B, T, dx)).astype(np.float32)
+    eye = np.eye(dx, dtype=np.float32)
+    Wt = np.stack([eye, 2 * eye, np.roll(eye, 1, axis=1)])               # row o of role v picks x[(o + 1) % dx]
+    Q, K, V = orc.project_qkv(X, Wt, H)
+    for h in range(H):
+        np.testing.assert_array_equal(Q[:, h], X[:, :, h * d:(h + 1) * d].astype(np.float64))
+        np.testing.assert_array_equal(K[:, h], 2.0 * X[:, :, h * d:(h + 1) * d].astype(np.float64))
+        cols = [(h * d + e + 1) % dx for e in range(d)]
+        np.testing.assert_array_equal(V[:, h], X[:, :, cols].astype(np.float64))
+    # a one-hot input row reads out one column of each transposed matrix: catches a transposed operand
+    X1 = np.zeros((1, 1, dx), dtype=np.float32)
+    X1[0, 0, 4] = 1.0
+    _, Wr = _proj_rand(1, 1, dx, H, d, 6)
+    out = orc.project_qkv(X1, Wr, H)
+    for r in range(3):
+        for h in range(H):
+            np.testing.assert_array_equal(out[r][0, h, 0], Wr[r, h * d:(h + 1) * d, 4].astype(np.float64))
+
+
+def test_projection_linearity_and_padding():
+    B, T, dx, H, d = 2, 6, 8, 2, 4
+    X, Wt = _proj_rand(B, T, dx, H, d, 21)
+    X2, _ = _proj_rand(B, T, dx, H, d, 22)
+    a = orc.project_qkv(X, Wt, H)
+    b = orc.project_qkv(X2, Wt, H)
+    s = orc.project_qkv((X.astype(np.float64) + 0.5 * X2).astype(np.float32), Wt, H)
+    for r in range(3):
+        np.testing.assert_allclose(s[r], a[r] + 0.5 * b[r], rtol=0, atol=2e-6)   # float32 rounding of the sum of inputs
+    lengths = np.array([3, 6], dtype=np.int32)
+    Xn = X.copy()
+    Xn[0, 3:] = np.nan                                                   # padded rows are never read
+    p = orc.project_qkv(Xn, Wt, H, lengths)
+    for r in range(3):
+        assert np.all(p[r][0, :, 3:] == 0.0)
+        np.testing.assert_array_equal(p[r][0, :, :3], a[r][0, :, :3])
+        np.testing.assert_array_equal(p[r][1], a[r][1])
+
+
+def test_projection_workload_generator():
+    w = wl.WORKLOADS["tiny_fp32"]
+    a, b = wl.make_projection_inputs(w), wl.make_projection_inputs(w)
+    assert a["X"].shape == (w.B, w.T, w.H * w.d) and a["Wt"].shape == (3, w.H * w.d, w.H * w.d)
+    np.testing.assert_array_equal(a["X"], b["X"])
+    np.testing.assert_array_equal(a["Wt"], b["Wt"])
+    Q, _, _ = orc.project_qkv(a["X"], a["Wt"], w.H)
+    assert 0.8 < Q.std() < 1.2                                           # unit-variance activations by construction

@@ -40,6 +40,15 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+def tensor_peak():
+    """Dense bf16 tensor throughput (TFLOP/s) for a kernel timed alone: the measured burst figure."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of the dominant kernel from the
 # ncu capture summarised under profiles/, valid only while the kernel's sources are unchanged.
 _FUSED_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.cuh", "psattn_select.cuh",
@@ -47,12 +56,12 @@ _FUSED_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.
 _STREAM_SOURCES = ["psattn_measure_mma.cu", "psattn_measure_stream.cuh", "psattn_measure_mma.cuh",
                    "psattn_sm100.cuh", "psattn_common.cuh"]
 TRAFFIC = {
-    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53704704, "sources": _FUSED_SOURCES,
+    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53888512, "sources": _FUSED_SOURCES,
                    "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
-                   "sources_sha1": "pending"},
-    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76376576, "sources": _STREAM_SOURCES,
+                   "sources_sha1": "e084895faff67566dc7d5a38fb4974b43d42098c"},
+    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76131840, "sources": _STREAM_SOURCES,
                   "profile": "profiles/ncu_full_k_measure_stream_long_bf16.txt",
-                  "sources_sha1": "pending"},
+                  "sources_sha1": "82ed0366c49abb6f65111aca1badde55122744b3"},
 }
 
 
@@ -413,6 +422,30 @@ def main():
         x_ms = time_events(exact, 5, torch)
         x_flops = 2.0 * w.d * sum(int(L) * int(L) for L in host_sets[0]["lengths"]) * w.H
         variants["exact_measure"] = {"ms_per_step": x_ms, "tflops": x_flops / (x_ms * 1e-3) / 1e12}
+        # Sec. 3.1: the projections in front of the path (one tcgen05 GEMM writing Q, K, V in the layout
+        # the path reads, plus mean(V)); reported against the measured dense bf16 peak
+        if w.dtype == "bf16":
+            dx = w.H * w.d
+            pin = wl.make_projection_inputs(w, seed=sharding.rank_seed(w.seed, rank, 0))
+            pX = [torch.from_numpy(pin["X"]).to("cuda", tdt) for _ in range(n_sets)]
+            pW = torch.from_numpy(pin["Wt"]).to("cuda", tdt)
+            vb = torch.empty((w.B, w.H, w.d), dtype=torch.float32, device="cuda")
+            pO = [[torch.empty((w.B, w.H, w.T, w.d), dtype=tdt, device="cuda") for _ in range(3)] for _ in range(n_sets)]
+
+            def project(k):
+                o = pO[k % n_sets]
+                plan.psattn_project_qkv(pX[k % n_sets], pW, sets[k % n_sets]["lengths"], o[0], o[1], o[2], vb)
+            r_pj = replayer(project, capture(project))
+            for k in range(3):
+                r_pj(k)
+            p_ms = time_events(r_pj, nk, torch, grouped=True)
+            p_flops = 2.0 * dx * 3 * dx * sum(int(L) for L in host_sets[0]["lengths"])
+            tf_peak = tensor_peak()
+            variants["qkv_projection"] = {
+                "ms_per_step": p_ms, "tflops": p_flops / (p_ms * 1e-3) / 1e12, "peak_tflops": tf_peak[0],
+                "frac_of_tensor_peak": p_flops / (p_ms * 1e-3) / 1e12 / tf_peak[0], "peak_kind": "of " + tf_peak[1],
+                "d_x": dx, "device_status": plan.psattn_read_status()}
+            del pO, pX
     peak, peak_kind = measured_peaks()
     units = w.B * w.H
     measure_bytes = units * w.T * w.d * elem * 2 + w.B * w.T * n_cols * 4 + units * w.T * 4

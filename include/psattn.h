@@ -143,6 +143,23 @@ int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K, const int3
 int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const void *K, const int32_t *lengths,
                          float *M_out, void *workspace, size_t workspace_bytes, void *stream);
 
+/* The projections that precede the attention (Sec. 3.1: "Q = X W_q, K = X W_k, V = X W_v"), for all heads
+ * at once, written directly in the layout the calls above read.  All pointers device.
+ *   X     [B][T_max][d_x], dense, element type of the plan (the layer input; d_x is the model width)
+ *   Wt    [3][H * 64][d_x], dense, same type: the matrices stored transposed, role r = 0 (q), 1 (k), 2 (v),
+ *         row h * 64 + e of role r = column e of head h's matrix: Wt[r][h*64 + e][x] = W_r^h[x][e]
+ *   Q, K, V  outputs of the plan's type with the descriptor's q/k/v strides:
+ *         Q[b][h][t][e] = sum_x X[b][t][x] W_q^h[x][e] (fp32 accumulation, rounded to the output type)
+ *         for t < lengths[b]; rows at positions >= lengths[b] are NOT written (the attention never reads them)
+ *   vbar  optional (may be NULL) fp32 [B][H][64]: mean over t < lengths[b] of V as stored, i.e. the fill
+ *         value of step (e), produced while V is written instead of by another pass over it
+ * bf16: a tcgen05 GEMM (d_x must be a multiple of 8; otherwise, for fp32, and with PSATTN_PATH_STAGED, a
+ * plain fp32-FMA kernel runs).  Base pointers 16-byte aligned.  Uses the workspace (stream-ordered with
+ * other calls on it). */
+int psattn_project_qkv(psattn_plan_t *plan, const void *X, const void *Wt, int32_t d_x,
+                       const int32_t *lengths, void *Q, void *K, void *V, float *vbar,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
 /* Step (c) only (Sec. 3.2): top-u positions of M (fp32 [B][H][T_max]) among i < lengths[b]. */
 int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
                   int32_t *sel_idx, void *workspace, size_t workspace_bytes, void *stream);

@@ -21,7 +21,7 @@ EXPORTS = [
     "psattn_plan_create", "psattn_plan_destroy", "psattn_plan_limits", "psattn_workspace_bytes",
     "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_exact_measure", "psattn_select",
     "psattn_mean_v", "psattn_attend_rows", "psattn_dense_forward", "psattn_read_status",
-    "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc",
+    "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc", "psattn_project_qkv",
 ]
 
 
@@ -75,6 +75,7 @@ def load(build_if_missing: bool = True):
     lib.psattn_measure.argtypes = [vp] * 7 + [sz, vp]
     lib.psattn_exact_measure.argtypes = [vp] * 6 + [sz, vp]
     lib.psattn_select.argtypes = [vp] * 5 + [sz, vp]
+    lib.psattn_project_qkv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.psattn_mean_v.argtypes = [vp] * 5 + [sz, vp]
     lib.psattn_attend_rows.argtypes = [vp] * 6 + [i32, vp, vp, sz, vp]
     lib.psattn_dense_forward.argtypes = [vp] * 7 + [sz, vp]
@@ -212,6 +213,20 @@ class Plan:
         _check(self.lib.psattn_exact_measure(self.handle, _ptr(Q), _ptr(K), _ptr(lengths), _ptr(M_out),
                                              ws, n, _stream()), self.handle)
         return M_out
+
+    def psattn_project_qkv(self, X, Wt, lengths=None, Q=None, K=None, V=None, vbar=None):
+        """Q, K, V = X W_q, X W_k, X W_v in the attention layout; X [B, T_max, d_x], Wt [3, H*64, d_x].
+        Rows at padded positions of freshly allocated outputs are zero (the kernel does not write them)."""
+        outs = []
+        for t in (Q, K, V):
+            if t is None:
+                t = torch.zeros((self.B, self.H, self.T_max, self.d_head), dtype=self.dtype, device=X.device)
+            outs.append(t)
+        ws, n = self._ws()
+        _check(self.lib.psattn_project_qkv(self.handle, _ptr(X), _ptr(Wt), int(X.shape[-1]), _ptr(lengths),
+                                           _ptr(outs[0]), _ptr(outs[1]), _ptr(outs[2]), _ptr(vbar), ws, n,
+                                           _stream()), self.handle)
+        return tuple(outs)
 
     def psattn_select(self, M, lengths, sel_idx=None):
         if sel_idx is None:

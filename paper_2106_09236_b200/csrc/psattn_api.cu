@@ -21,7 +21,7 @@ struct psattn_plan {
     int *d_tables;                // device: u_tab[T+1] then U_tab[T+1]
     int last_cuda_error;
     // workspace layout (byte offsets)
-    size_t off_status, off_M, off_vpart, off_vbar, off_ml, off_acc, off_sel, ws_bytes;
+    size_t off_status, off_M, off_vpart, off_vbar, off_ml, off_acc, off_sel, off_pvsum, ws_bytes;
     // host-io staging (psattn_plan_enable_host_io)
     bool host_io;
     void *h_Q, *h_K, *h_V, *h_O, *h_ws;
@@ -155,6 +155,8 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     p->off_ml = off;     off = align_up(off + units * (u_max + 1) * p->n_splits * 2 * sizeof(float), 256);
     p->off_acc = off;    off = align_up(off + units * (u_max + 1) * p->n_splits * kD * sizeof(float), 256);
     p->off_sel = off;    off = align_up(off + units * u_max * sizeof(int), 256);
+    // per-tile column sums of V written by the projection kernel
+    p->off_pvsum = off;  off = align_up(off + project_vpart_floats(d.B, d.H, d.T_max) * sizeof(float), 256);
     p->ws_bytes = off;
     *out = p;
     return PSATTN_OK;
@@ -404,6 +406,21 @@ extern "C" int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const vo
     // PSATTN_PATH_STAGED keeps the arithmetic off the tensor cores (one warp per query)
     const int dtype = d.dtype == PSATTN_BF16 && d.path == PSATTN_PATH_STAGED ? 2 : d.dtype;
     PSATTN_CU(launch_exact_measure(dtype, g, Q, K, M_out, static_cast<cudaStream_t>(stream)));
+    return PSATTN_OK;
+}
+
+extern "C" int psattn_project_qkv(psattn_plan_t *plan, const void *X, const void *Wt, int32_t d_x,
+                                  const int32_t *lengths, void *Q, void *K, void *V, float *vbar,
+                                  void *workspace, size_t workspace_bytes, void *stream) {
+    if (!plan || !X || !Wt || !Q || !K || !V) return PSATTN_ERR_NULL;
+    if (d_x < 1 || d_x > (1 << 20)) return PSATTN_ERR_BAD_DESC;
+    if (!aligned16(X) || !aligned16(Wt) || !aligned16(Q) || !aligned16(K) || !aligned16(V)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    const psattn_desc_t &d = plan->desc;
+    Geom g = make_geom(plan, lengths, workspace);
+    PSATTN_CU(launch_project_qkv(d.dtype, d.path == PSATTN_PATH_STAGED, g, d_x, X, Wt, Q, K, V, vbar,
+                                 ws_at<float>(workspace, plan->off_pvsum), static_cast<cudaStream_t>(stream)));
     return PSATTN_OK;
 }
 

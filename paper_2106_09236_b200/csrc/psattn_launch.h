@@ -69,6 +69,12 @@ cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows,
                                 int n_splits, const float *part_ml, const float *part_acc, void *out,
                                 long long out_unit_stride, long long out_row_stride, int out_by_position,
                                 float *vbar, cudaStream_t st);
+// Sec. 3.1's projections Q = X W_q, K = X W_k, V = X W_v into the attention layout (tcgen05 GEMM for bf16,
+// dtype 0; one thread per element for fp32 or with force_simt).  X [B][T][dx], Wt [3][H*64][dx].
+// vbar (optional): mean(V) fp32 [B][H][64]; vpart: scratch of project_vpart_floats(B, H, T) floats.
+size_t project_vpart_floats(int B, int H, int T);
+cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx, const void *X, const void *Wt, void *Q,
+                               void *K, void *V, float *vbar, float *vpart, cudaStream_t st);
 cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
                         void *O, int own_v, cudaStream_t st);
 

@@ -1,0 +1,355 @@
+// The projections that precede the attention (Sec. 3.1): Q = X W_q, K = X W_k, V = X W_v, one
+// (d_x x 64) matrix per head and role, written straight into the [B][H][T][64] layout (any b/h/t strides)
+// that the attention kernels read, so no transpose pass sits between the two.
+//
+// bf16: ONE persistent tcgen05 GEMM over all three roles.  A tile is 128 tokens of one sequence x 256 output
+// columns (four 64-wide head blocks); CTAs walk the tiles round-robin.  Warp 0 streams 64-deep slabs of X and
+// of the transposed weights into a 4-stage shared-memory ring by TMA (128-byte swizzle), warp 1 issues
+// tcgen05.mma (M = 128, N = 256, K = 16) into one of two TMEM accumulators, warps 2-5 drain the other
+// accumulator: TMEM -> registers -> bf16 -> 128-byte row stores at (b, h, t).  The mainloop of tile i + 1 runs
+// under the drain of tile i.  Tiles that lie wholly beyond a sequence's length are skipped; rows beyond it
+// are not written.  For the V blocks the drain also reduces its 128 rows (as rounded to bf16) to one column
+// sum per block, in a fixed order, from which mean(V) - the fill value of step (e) - follows without
+// another pass over V.
+// fp32 (and layouts without a tensor map): one thread per output element, fp32 FMA.
+#include "psattn_launch.h"
+#include "psattn_sm100.cuh"
+
+namespace psattn {
+
+using namespace sm100;
+
+constexpr int kPjM = 128, kPjN = 256, kPjK = 64, kPjStages = 4;
+constexpr uint32_t kPjBytesA = kPjM * kPjK * 2, kPjBytesB = kPjN * kPjK * 2, kPjStage = kPjBytesA + kPjBytesB;
+constexpr uint32_t kPjOffBar = kPjStages * kPjStage;           // mbarriers, TMEM slot, abort flag
+constexpr uint32_t kPjOffRed = kPjOffBar + 128;                // [4 warps][64] column-sum staging
+constexpr uint32_t kPjSmem = kPjOffRed + 4 * 64 * 4;
+constexpr int kPjThreads = 192;
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
+
+struct ProjArgs {
+    int B, H, T, dx;
+    int tiles_per_seq, n_tiles_n, n_tiles;        // 128-token tiles per sequence, 256-column tiles, all tiles
+    long long qs[3], ks[3], vs[3];                // element strides (b, h, t) of the three outputs
+    __nv_bfloat16 *Q, *K, *V;
+    const int *lengths;
+    float *vpart;                                 // [B][tiles_per_seq][H][64] column sums of V per tile, or null
+    unsigned *status;
+};
+
+__device__ __forceinline__ int proj_len(const ProjArgs &a, int b) {
+    if (!a.lengths) return a.T;
+    int L = a.lengths[b];
+    if (L < 0 || L > a.T) {
+        atomicOr(a.status, kStatusLenClamped);
+        L = L < 0 ? 0 : a.T;
+    }
+    return L;
+}
+
+__global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const __grid_constant__ CUtensorMap tmX,
+                                                               const __grid_constant__ CUtensorMap tmW) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + kPjOffBar), *empty = full + kPjStages;
+    uint64_t *acc_full = empty + kPjStages, *acc_empty = acc_full + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    float *red = reinterpret_cast<float *>(smem + kPjOffRed);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if ((smem_u32(smem) & 1023u) != 0u) {                      // swizzled tiles need a 1024-byte base
+        if (tid == 0) atomicOr(a.status, kStatusWaitExpired);
+        return;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kPjStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&acc_full[s], 1); mbar_init(&acc_empty[s], 4); }
+        *abort_flag = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmW);
+    }
+    __syncwarp();
+    if (warp == 1) tmem_alloc(tmem_slot, 512);                 // two accumulators of 256 columns
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int n_kb = (a.dx + kPjK - 1) / kPjK;
+
+    if (warp == 0) {
+        // ---- producer: one lane streams the slabs of every tile of this CTA through the ring ----
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int tile = blockIdx.x; tile < a.n_tiles && !*abort_flag; tile += gridDim.x) {
+                const int n = tile % a.n_tiles_n, m = tile / a.n_tiles_n;
+                const int b = m / a.tiles_per_seq, tt = m % a.tiles_per_seq;
+                if (tt * kPjM >= proj_len(a, b)) continue;
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    const uint32_t s = it % kPjStages, ph = (it / kPjStages) & 1u;
+                    if (!mbar_wait(&empty[s], ph ^ 1u)) { atomicOr(a.status, kStatusWaitExpired); *abort_flag = 1; break; }
+                    uint8_t *sa = smem + s * kPjStage;
+                    mbar_expect_tx(&full[s], kPjStage);
+                    tma_load_3d(sa, &tmX, &full[s], kb * kPjK, tt * kPjM, b);
+                    tma_load_2d(sa + kPjBytesA, &tmW, &full[s], kb * kPjK, n * kPjN);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer: one lane; accumulator (tile count & 1) ----
+        if (lane == 0) {
+            constexpr uint32_t kIdesc = umma_idesc_bf16(kPjM, kPjN, 0);
+            uint32_t it = 0, tc = 0;
+            for (int tile = blockIdx.x; tile < a.n_tiles && !*abort_flag; tile += gridDim.x) {
+                const int m = tile / a.n_tiles_n;
+                const int b = m / a.tiles_per_seq, tt = m % a.tiles_per_seq;
+                if (tt * kPjM >= proj_len(a, b)) continue;
+                const uint32_t acc = tc & 1u, aph = (tc >> 1) & 1u;
+                if (!mbar_wait(&acc_empty[acc], aph ^ 1u)) { atomicOr(a.status, kStatusWaitExpired); *abort_flag = 1; break; }
+                tc_fence_after();
+                bool ok = true;
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    const uint32_t s = it % kPjStages, ph = (it / kPjStages) & 1u;
+                    if (!mbar_wait(&full[s], ph)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + s * kPjStage), sb = sa + kPjBytesA;
+#pragma unroll
+                    for (int k = 0; k < kPjK / 16; ++k)
+                        umma_bf16(tmem_base + acc * kPjN, umma_desc_sw128(sa + k * 32, 16, 1024),
+                                  umma_desc_sw128(sb + k * 32, 16, 1024), kIdesc, (kb | k) != 0);
+                    umma_commit(&empty[s]);                    // the stage is free once these products have run
+                }
+                if (!ok) { atomicOr(a.status, kStatusWaitExpired); *abort_flag = 1; break; }
+                umma_commit(&acc_full[acc]);
+                ++tc;
+            }
+        }
+    } else {
+        // ---- drain: warp w reads TMEM lanes 32 (w % 4) .. + 31; thread = one token row ----
+        const int quarter = warp & 3, row = quarter * 32 + lane;
+        const int ew = warp - 2;                               // 0..3: slot in the column-sum staging
+        uint32_t tc = 0;
+        for (int tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
+            const int n = tile % a.n_tiles_n, m = tile / a.n_tiles_n;
+            const int b = m / a.tiles_per_seq, tt = m % a.tiles_per_seq;
+            const int L = proj_len(a, b);
+            if (tt * kPjM >= L) continue;
+            const uint32_t acc = tc & 1u, aph = (tc >> 1) & 1u;
+            const bool mine = !*abort_flag && mbar_wait(&acc_full[acc], aph);
+            uint32_t landed;                                   // the four drain warps decide together (they meet at
+            asm volatile(                                      // barrier 1 below, so none may leave alone)
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "bar.red.and.pred p, 1, 128, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(landed)
+                : "r"(mine ? 1u : 0u)
+                : "memory");
+            if (!landed) {
+                if (lane == 0) { atomicOr(a.status, kStatusWaitExpired); *abort_flag = 1; }
+                break;
+            }
+            tc_fence_after();
+            const int t = tt * kPjM + row;
+            const bool valid = t < L;
+#pragma unroll 1
+            for (int cc = 0; cc < kPjN / 64; ++cc) {
+                const int gc = n * (kPjN / 64) + cc;           // 64-column block: role = gc / H, head = gc % H
+                if (gc >= 3 * a.H) break;
+                const int role = gc / a.H, h = gc - role * a.H;
+                uint32_t r0[32], r1[32];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kPjN + cc * 64;
+                tmem_ld32_issue(taddr, r0);
+                tmem_ld32_issue(taddr + 32, r1);
+                tmem_ld_wait();
+                tmem_ld_fence32(r0);
+                tmem_ld_fence32(r1);
+                uint32_t pk[32];                               // 64 bf16, two per word
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    __nv_bfloat162 p = __floats2bfloat162_rn(__uint_as_float(r0[2 * j]), __uint_as_float(r0[2 * j + 1]));
+                    __nv_bfloat162 q = __floats2bfloat162_rn(__uint_as_float(r1[2 * j]), __uint_as_float(r1[2 * j + 1]));
+                    pk[j] = *reinterpret_cast<uint32_t *>(&p);
+                    pk[16 + j] = *reinterpret_cast<uint32_t *>(&q);
+                }
+                if (valid) {
+                    const long long *st = role == 0 ? a.qs : (role == 1 ? a.ks : a.vs);
+                    __nv_bfloat16 *base = role == 0 ? a.Q : (role == 1 ? a.K : a.V);
+                    uint4 *dst = reinterpret_cast<uint4 *>(base + (long long)b * st[0] + (long long)h * st[1] + (long long)t * st[2]);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                }
+                if (role == 2 && a.vpart != nullptr) {
+                    // column sums of this block over the tile's valid rows, from the values as stored (bf16)
+                    float v[64];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        v[2 * j] = valid ? __uint_as_float(pk[j] << 16) : 0.f;
+                        v[2 * j + 1] = valid ? __uint_as_float(pk[j] & 0xffff0000u) : 0.f;
+                    }
+                    // transposing butterfly: after the step with offset o a lane keeps half of its columns;
+                    // at the end lane l holds the sums of columns 2 l and 2 l + 1 over the warp's 32 rows
+#pragma unroll
+                    for (int o = 16, cnt = 32; o >= 1; o >>= 1, cnt >>= 1) {
+                        const bool up = (lane & o) != 0;
+#pragma unroll
+                        for (int i = 0; i < cnt; ++i) {
+                            const float send = up ? v[i] : v[i + cnt];
+                            const float keep = up ? v[i + cnt] : v[i];
+                            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                        }
+                    }
+                    red[ew * 64 + 2 * lane] = v[0];
+                    red[ew * 64 + 2 * lane + 1] = v[1];
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int et = tid - 64;                   // 0..127 within the drain warps
+                    if (et < 64) {
+                        // rows 0-31 are drained by warp 4 (slot 2), 32-63 by warp 5, 64-95 by warp 2, 96-127 by warp 3
+                        const float s = ((red[2 * 64 + et] + red[3 * 64 + et]) + red[0 * 64 + et]) + red[1 * 64 + et];
+                        a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + et] = s;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[acc]);
+            ++tc;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+// mean(V) of every unit from the per-tile column sums, in tile order.
+__global__ void __launch_bounds__(64) k_project_vbar(ProjArgs a, float *__restrict__ vbar) {
+    const int unit = blockIdx.x, b = unit / a.H, h = unit % a.H, e = threadIdx.x;
+    const int L = proj_len(a, b);
+    float s = 0.f;
+    for (int tt = 0; tt * kPjM < L; ++tt) s += a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + e];
+    vbar[(long long)unit * 64 + e] = L > 0 ? s / (float)L : 0.f;
+}
+
+// Any element type and layout: one thread per output element (64 threads = one head block of one token).
+template <typename DT>
+__global__ void __launch_bounds__(64) k_project_simt(ProjArgs a, const DT *__restrict__ X, const DT *__restrict__ Wt,
+                                                     DT *Q, DT *K, DT *V) {
+    const int e = threadIdx.x, gc = blockIdx.y;
+    const int b = blockIdx.x / a.T, t = blockIdx.x % a.T;
+    if (t >= proj_len(a, b)) return;
+    const int role = gc / a.H, h = gc - role * a.H;
+    const DT *x = X + ((long long)b * a.T + t) * a.dx;
+    const DT *w = Wt + ((long long)gc * 64 + e) * a.dx;
+    float acc = 0.f;
+    for (int k = 0; k < a.dx; ++k) acc = fmaf((float)x[k], (float)w[k], acc);
+    const long long *st = role == 0 ? a.qs : (role == 1 ? a.ks : a.vs);
+    DT *base = role == 0 ? Q : (role == 1 ? K : V);
+    base[(long long)b * st[0] + (long long)h * st[1] + (long long)t * st[2] + e] = (DT)acc;
+}
+
+// mean(V) from the stored V (SIMT path): one block per unit, fixed order over t.
+template <typename DT>
+__global__ void __launch_bounds__(64) k_project_vbar_simt(ProjArgs a, const DT *__restrict__ V, float *__restrict__ vbar) {
+    const int unit = blockIdx.x, b = unit / a.H, h = unit % a.H, e = threadIdx.x;
+    const int L = proj_len(a, b);
+    const DT *v = V + (long long)b * a.vs[0] + (long long)h * a.vs[1] + e;
+    float s = 0.f;
+    for (int t = 0; t < L; ++t) s += (float)v[(long long)t * a.vs[2]];
+    vbar[(long long)unit * 64 + e] = L > 0 ? s / (float)L : 0.f;
+}
+
+typedef CUresult (*EncodeTiledFnP)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+static EncodeTiledFnP proj_encode_fn() {
+    static EncodeTiledFnP fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFnP>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+size_t project_vpart_floats(int B, int H, int T) { return (size_t)B * ((T + kPjM - 1) / kPjM) * H * 64; }
+
+// dtype 0 = bf16, 1 = fp32.  X [B][T][dx], Wt [3][H*64][dx], outputs with g.qs / g.ks / g.vs strides.
+// vbar (optional) fp32 [B][H][64]; vpart = scratch of project_vpart_floats() floats (needed with vbar on the
+// tensor-core path).  force_simt keeps bf16 inputs off the tensor cores.
+cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx, const void *X, const void *Wt, void *Q,
+                               void *K, void *V, float *vbar, float *vpart, cudaStream_t st) {
+    if (g.B * g.H == 0) return cudaSuccess;
+    ProjArgs a;
+    a.B = g.B; a.H = g.H; a.T = g.T; a.dx = dx;
+    a.tiles_per_seq = (g.T + kPjM - 1) / kPjM;
+    a.n_tiles_n = (3 * g.H * 64 + kPjN - 1) / kPjN;
+    a.n_tiles = g.B * a.tiles_per_seq * a.n_tiles_n;
+    for (int k = 0; k < 3; ++k) { a.qs[k] = g.qs[k]; a.ks[k] = g.ks[k]; a.vs[k] = g.vs[k]; }
+    a.Q = (__nv_bfloat16 *)Q; a.K = (__nv_bfloat16 *)K; a.V = (__nv_bfloat16 *)V;
+    a.lengths = g.lengths; a.status = g.status;
+    a.vpart = vbar ? vpart : nullptr;
+    EncodeTiledFnP enc = proj_encode_fn();
+    if (dtype == 0 && !force_simt && enc && dx % 8 == 0 && (vbar == nullptr || vpart != nullptr)) {
+        CUtensorMap tmX, tmW;
+        const cuuint64_t xdim[3] = {(cuuint64_t)dx, (cuuint64_t)g.T, (cuuint64_t)g.B};
+        const cuuint64_t xstr[2] = {(cuuint64_t)dx * 2, (cuuint64_t)g.T * dx * 2};
+        const cuuint32_t xbox[3] = {kPjK, kPjM, 1}, one3[3] = {1, 1, 1};
+        const cuuint64_t wdim[2] = {(cuuint64_t)dx, (cuuint64_t)3 * g.H * 64};
+        const cuuint64_t wstr[1] = {(cuuint64_t)dx * 2};
+        const cuuint32_t wbox[2] = {kPjK, kPjN}, one2[2] = {1, 1};
+        const bool ok =
+            enc(&tmX, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(X), xdim, xstr, xbox, one3,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS &&
+            enc(&tmW, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(Wt), wdim, wstr, wbox, one2,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        if (ok) {
+            static bool attr_set = false;
+            if (!attr_set) {
+                cudaError_t e = cudaFuncSetAttribute(k_project_qkv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPjSmem);
+                if (e != cudaSuccess) return e;
+                attr_set = true;
+            }
+            const int grid = a.n_tiles < kSmCount ? a.n_tiles : kSmCount;
+            k_project_qkv<<<grid, kPjThreads, kPjSmem, st>>>(a, tmX, tmW);
+            note_launch();
+            cudaError_t e = cudaGetLastError();
+            if (e != cudaSuccess || vbar == nullptr) return e;
+            k_project_vbar<<<g.B * g.H, 64, 0, st>>>(a, vbar);
+            note_launch();
+            return cudaGetLastError();
+        }
+    }
+    const dim3 grid((unsigned)(g.B * g.T), (unsigned)(3 * g.H));
+    if (dtype == 0) {
+        k_project_simt<__nv_bfloat16><<<grid, 64, 0, st>>>(a, (const __nv_bfloat16 *)X, (const __nv_bfloat16 *)Wt,
+                                                            (__nv_bfloat16 *)Q, (__nv_bfloat16 *)K, (__nv_bfloat16 *)V);
+        note_launch();
+        if (vbar) { k_project_vbar_simt<__nv_bfloat16><<<g.B * g.H, 64, 0, st>>>(a, (const __nv_bfloat16 *)V, vbar); note_launch(); }
+    } else {
+        k_project_simt<float><<<grid, 64, 0, st>>>(a, (const float *)X, (const float *)Wt, (float *)Q, (float *)K, (float *)V);
+        note_launch();
+        if (vbar) { k_project_vbar_simt<float><<<g.B * g.H, 64, 0, st>>>(a, (const float *)V, vbar); note_launch(); }
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace psattn

@@ -432,19 +432,21 @@ def main():
             vb = torch.empty((w.B, w.H, w.d), dtype=torch.float32, device="cuda")
             pO = [[torch.empty((w.B, w.H, w.T, w.d), dtype=tdt, device="cuda") for _ in range(3)] for _ in range(n_sets)]
 
-            def project(k):
-                o = pO[k % n_sets]
-                plan.psattn_project_qkv(pX[k % n_sets], pW, sets[k % n_sets]["lengths"], o[0], o[1], o[2], vb)
-            r_pj = replayer(project, capture(project))
-            for k in range(3):
-                r_pj(k)
-            p_ms = time_events(r_pj, nk, torch, grouped=True)
             p_flops = 2.0 * dx * 3 * dx * sum(int(L) for L in host_sets[0]["lengths"])
             tf_peak = tensor_peak()
-            variants["qkv_projection"] = {
-                "ms_per_step": p_ms, "tflops": p_flops / (p_ms * 1e-3) / 1e12, "peak_tflops": tf_peak[0],
-                "frac_of_tensor_peak": p_flops / (p_ms * 1e-3) / 1e12 / tf_peak[0], "peak_kind": "of " + tf_peak[1],
-                "d_x": dx, "device_status": plan.psattn_read_status()}
+            for key, want_vbar in (("qkv_projection", True), ("qkv_projection_without_mean_v", False)):
+                def project(k, want_vbar=want_vbar):
+                    o = pO[k % n_sets]
+                    plan.psattn_project_qkv(pX[k % n_sets], pW, sets[k % n_sets]["lengths"], o[0], o[1], o[2],
+                                            vb if want_vbar else None)
+                r_pj = replayer(project, capture(project))
+                for k in range(3):
+                    r_pj(k)
+                p_ms = time_events(r_pj, nk, torch, grouped=True)
+                variants[key] = {
+                    "ms_per_step": p_ms, "tflops": p_flops / (p_ms * 1e-3) / 1e12, "peak_tflops": tf_peak[0],
+                    "frac_of_tensor_peak": p_flops / (p_ms * 1e-3) / 1e12 / tf_peak[0],
+                    "peak_kind": "of " + tf_peak[1], "d_x": dx, "device_status": plan.psattn_read_status()}
             del pO, pX
     peak, peak_kind = measured_peaks()
     units = w.B * w.H

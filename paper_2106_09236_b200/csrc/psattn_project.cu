@@ -2,11 +2,11 @@
 // (d_x x 64) matrix per head and role, written straight into the [B][H][T][64] layout (any b/h/t strides)
 // that the attention kernels read, so no transpose pass sits between the two.
 //
-// bf16: ONE persistent tcgen05 GEMM over all three roles.  A tile is 128 tokens of one sequence x 256 output
-// columns (four 64-wide head blocks); CTAs walk the tiles round-robin.  Warp 0 streams 64-deep slabs of X and
-// of the transposed weights into a 4-stage shared-memory ring by TMA (128-byte swizzle), warp 1 issues
-// tcgen05.mma (M = 128, N = 256, K = 16) into one of two TMEM accumulators, warps 2-5 drain the other
-// accumulator: TMEM -> registers -> bf16 -> 128-byte row stores at (b, h, t).  The mainloop of tile i + 1 runs
+// bf16: ONE persistent tcgen05 GEMM over all three roles.  A tile is 128 tokens of one sequence x 192 output
+// columns (three 64-wide head blocks); CTAs walk the tiles round-robin.  Warp 0 streams 64-deep slabs of X and
+// of the transposed weights into a 5-stage shared-memory ring by TMA (128-byte swizzle), warp 1 issues
+// tcgen05.mma (M = 128, N = 192, K = 16) into one of two TMEM accumulators, warps 2-5 drain the other
+// accumulator: TMEM -> registers -> bf16 -> a swizzled staging tile -> whole 128-byte rows at (b, h, t).  The mainloop of tile i + 1 runs
 // under the drain of tile i.  Tiles that lie wholly beyond a sequence's length are skipped; rows beyond it
 // are not written.  For the V blocks the drain also reduces its 128 rows (as rounded to bf16) to one column
 // sum per block, in a fixed order, from which mean(V) - the fill value of step (e) - follows without
@@ -19,11 +19,13 @@ namespace psattn {
 
 using namespace sm100;
 
-constexpr int kPjM = 128, kPjN = 256, kPjK = 64, kPjStages = 4;
+constexpr int kPjM = 128, kPjN = 192, kPjK = 64, kPjStages = 5;
+constexpr int kPjAccCols = 256;                                // TMEM columns reserved per accumulator
 constexpr uint32_t kPjBytesA = kPjM * kPjK * 2, kPjBytesB = kPjN * kPjK * 2, kPjStage = kPjBytesA + kPjBytesB;
 constexpr uint32_t kPjOffBar = kPjStages * kPjStage;           // mbarriers, TMEM slot, abort flag
 constexpr uint32_t kPjOffRed = kPjOffBar + 128;                // [4 warps][64] column-sum staging
-constexpr uint32_t kPjSmem = kPjOffRed + 4 * 64 * 4;
+constexpr uint32_t kPjOffStage = kPjOffRed + 4 * 64 * 4;       // [4 warps][32 rows][128 B] output staging (swizzled)
+constexpr uint32_t kPjSmem = kPjOffStage + 4 * 4096;
 constexpr int kPjThreads = 192;
 
 __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *m, uint64_t *bar, int c0, int c1) {
@@ -39,7 +41,7 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *m, uin
 
 struct ProjArgs {
     int B, H, T, dx;
-    int tiles_per_seq, n_tiles_n, n_tiles;        // 128-token tiles per sequence, 256-column tiles, all tiles
+    int tiles_per_seq, n_tiles_n, n_tiles;        // 128-token tiles per sequence, 192-column tiles, all tiles
     long long qs[3], ks[3], vs[3];                // element strides (b, h, t) of the three outputs
     __nv_bfloat16 *Q, *K, *V;
     const int *lengths;
@@ -78,10 +80,14 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
         tma_prefetch_desc(&tmX); tma_prefetch_desc(&tmW);
     }
     __syncwarp();
-    if (warp == 1) tmem_alloc(tmem_slot, 512);                 // two accumulators of 256 columns
+    // programmatic dependent launch: the next kernel of the stream may be scheduled now (it waits at its own
+    // griddepcontrol.wait); nothing in global memory is touched before the previous grid has completed
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (warp == 1) tmem_alloc(tmem_slot, 512);                 // two accumulators, 192 of 256 columns each
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     const int n_kb = (a.dx + kPjK - 1) / kPjK;
 
@@ -123,7 +129,7 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
                     const uint32_t sa = smem_u32(smem + s * kPjStage), sb = sa + kPjBytesA;
 #pragma unroll
                     for (int k = 0; k < kPjK / 16; ++k)
-                        umma_bf16(tmem_base + acc * kPjN, umma_desc_sw128(sa + k * 32, 16, 1024),
+                        umma_bf16(tmem_base + acc * kPjAccCols, umma_desc_sw128(sa + k * 32, 16, 1024),
                                   umma_desc_sw128(sb + k * 32, 16, 1024), kIdesc, (kb | k) != 0);
                     umma_commit(&empty[s]);                    // the stage is free once these products have run
                 }
@@ -135,7 +141,8 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
     } else {
         // ---- drain: warp w reads TMEM lanes 32 (w % 4) .. + 31; thread = one token row ----
         const int quarter = warp & 3, row = quarter * 32 + lane;
-        const int ew = warp - 2;                               // 0..3: slot in the column-sum staging
+        const int ew = warp - 2;                               // 0..3: slot in the staging buffers
+        uint4 *stage = reinterpret_cast<uint4 *>(smem + kPjOffStage + ew * 4096);
         uint32_t tc = 0;
         for (int tile = blockIdx.x; tile < a.n_tiles; tile += gridDim.x) {
             const int n = tile % a.n_tiles_n, m = tile / a.n_tiles_n;
@@ -160,33 +167,36 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
             tc_fence_after();
             const int t = tt * kPjM + row;
             const bool valid = t < L;
-#pragma unroll 1
-            for (int cc = 0; cc < kPjN / 64; ++cc) {
-                const int gc = n * (kPjN / 64) + cc;           // 64-column block: role = gc / H, head = gc % H
-                if (gc >= 3 * a.H) break;
+            const int n_cc = min(kPjN / 64, 3 * a.H - n * (kPjN / 64));   // 64-column blocks of this tile
+            const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kPjAccCols;
+            uint32_t ra[64], rb[64];                           // two blocks in flight: the next one loads while
+            tmem_ld32_issue(tacc, ra);                         // the current one is converted and stored
+            tmem_ld32_issue(tacc + 32, ra + 32);
+            auto drain_block = [&](uint32_t (&r)[64], int cc) {
+                const int gc = n * (kPjN / 64) + cc;           // role = gc / H, head = gc % H
                 const int role = gc / a.H, h = gc - role * a.H;
-                uint32_t r0[32], r1[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kPjN + cc * 64;
-                tmem_ld32_issue(taddr, r0);
-                tmem_ld32_issue(taddr + 32, r1);
-                tmem_ld_wait();
-                tmem_ld_fence32(r0);
-                tmem_ld_fence32(r1);
                 uint32_t pk[32];                               // 64 bf16, two per word
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    __nv_bfloat162 p = __floats2bfloat162_rn(__uint_as_float(r0[2 * j]), __uint_as_float(r0[2 * j + 1]));
-                    __nv_bfloat162 q = __floats2bfloat162_rn(__uint_as_float(r1[2 * j]), __uint_as_float(r1[2 * j + 1]));
-                    pk[j] = *reinterpret_cast<uint32_t *>(&p);
-                    pk[16 + j] = *reinterpret_cast<uint32_t *>(&q);
+                for (int j = 0; j < 32; ++j) {
+                    __nv_bfloat162 p2 = __floats2bfloat162_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+                    pk[j] = *reinterpret_cast<uint32_t *>(&p2);
                 }
-                if (valid) {
-                    const long long *st = role == 0 ? a.qs : (role == 1 ? a.ks : a.vs);
-                    __nv_bfloat16 *base = role == 0 ? a.Q : (role == 1 ? a.K : a.V);
-                    uint4 *dst = reinterpret_cast<uint4 *>(base + (long long)b * st[0] + (long long)h * st[1] + (long long)t * st[2]);
+                // through a swizzled staging tile, so that each store instruction of the warp writes four
+                // whole 128-byte rows instead of 16 bytes of 32 different rows
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                for (int j = 0; j < 8; ++j)
+                    stage[lane * 8 + (j ^ (lane & 7))] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                __syncwarp();
+                const long long *st = role == 0 ? a.qs : (role == 1 ? a.ks : a.vs);
+                __nv_bfloat16 *base = (role == 0 ? a.Q : (role == 1 ? a.K : a.V)) + (long long)b * st[0] + (long long)h * st[1];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = 4 * i + (lane >> 3), c = lane & 7;
+                    const int tr = tt * kPjM + quarter * 32 + rr;
+                    const uint4 val = stage[rr * 8 + (c ^ (rr & 7))];
+                    if (tr < L) reinterpret_cast<uint4 *>(base + (long long)tr * st[2])[c] = val;
                 }
+                __syncwarp();
                 if (role == 2 && a.vpart != nullptr) {
                     // column sums of this block over the tile's valid rows, from the values as stored (bf16)
                     float v[64];
@@ -213,10 +223,25 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
                     const int et = tid - 64;                   // 0..127 within the drain warps
                     if (et < 64) {
                         // rows 0-31 are drained by warp 4 (slot 2), 32-63 by warp 5, 64-95 by warp 2, 96-127 by warp 3
-                        const float s = ((red[2 * 64 + et] + red[3 * 64 + et]) + red[0 * 64 + et]) + red[1 * 64 + et];
-                        a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + et] = s;
+                        const float sum = ((red[2 * 64 + et] + red[3 * 64 + et]) + red[0 * 64 + et]) + red[1 * 64 + et];
+                        a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + et] = sum;
                     }
                     asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+            };
+#pragma unroll
+            for (int cc = 0; cc < kPjN / 64; cc += 2) {
+                if (cc < n_cc) {
+                    tmem_ld_wait();
+                    tmem_ld_fence32(ra); tmem_ld_fence32(ra + 32);
+                    if (cc + 1 < n_cc) { tmem_ld32_issue(tacc + (cc + 1) * 64, rb); tmem_ld32_issue(tacc + (cc + 1) * 64 + 32, rb + 32); }
+                    drain_block(ra, cc);
+                }
+                if (cc + 1 < n_cc) {
+                    tmem_ld_wait();
+                    tmem_ld_fence32(rb); tmem_ld_fence32(rb + 32);
+                    if (cc + 2 < n_cc) { tmem_ld32_issue(tacc + (cc + 2) * 64, ra); tmem_ld32_issue(tacc + (cc + 2) * 64 + 32, ra + 32); }
+                    drain_block(rb, cc + 1);
                 }
             }
             tc_fence_before();
@@ -233,6 +258,8 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
 // mean(V) of every unit from the per-tile column sums, in tile order.
 __global__ void __launch_bounds__(64) k_project_vbar(ProjArgs a, float *__restrict__ vbar) {
     const int unit = blockIdx.x, b = unit / a.H, h = unit % a.H, e = threadIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");        // the per-tile sums of the kernel before
     const int L = proj_len(a, b);
     float s = 0.f;
     for (int tt = 0; tt * kPjM < L; ++tt) s += a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + e];
@@ -328,14 +355,27 @@ cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx,
                 if (e != cudaSuccess) return e;
                 attr_set = true;
             }
-            const int grid = a.n_tiles < kSmCount ? a.n_tiles : kSmCount;
-            k_project_qkv<<<grid, kPjThreads, kPjSmem, st>>>(a, tmX, tmW);
+            // both kernels carry a programmatic dependency on their predecessor in the stream
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(a.n_tiles < kSmCount ? a.n_tiles : kSmCount));
+            cfg.blockDim = dim3(kPjThreads);
+            cfg.dynamicSmemBytes = kPjSmem;
+            cfg.stream = st;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cudaError_t e = cudaLaunchKernelEx(&cfg, k_project_qkv, a, tmX, tmW);
             note_launch();
-            cudaError_t e = cudaGetLastError();
+            if (e == cudaSuccess) e = cudaGetLastError();
             if (e != cudaSuccess || vbar == nullptr) return e;
-            k_project_vbar<<<g.B * g.H, 64, 0, st>>>(a, vbar);
+            cfg.gridDim = dim3((unsigned)(g.B * g.H));
+            cfg.blockDim = dim3(64);
+            cfg.dynamicSmemBytes = 0;
+            e = cudaLaunchKernelEx(&cfg, k_project_vbar, a, vbar);
             note_launch();
-            return cudaGetLastError();
+            return e != cudaSuccess ? e : cudaGetLastError();
         }
     }
     const dim3 grid((unsigned)(g.B * g.T), (unsigned)(3 * g.H));

@@ -198,6 +198,39 @@ def test_run_to_run_determinism(path):
 
 
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
+@pytest.mark.parametrize("dtype,T", [("bf16", 300), ("bf16", 1500), ("fp32", 200)])
+def test_workspace_contents_do_not_matter_and_its_bounds_are_kept(dtype, T, path):
+    """The scratch beyond the status word needs no initialisation: a run on a workspace full of 0xFF bytes
+    (NaN as floats, -1 as indices) gives bit-identical results, and the bytes on either side of the
+    workspace are not touched."""
+    B, H, c = 3, 2, 5.0
+    n = max(orc.count(c, L) for L in range(1, T + 1))
+    inp = _synth(B, H, T, 900 + T, n, dtype, [T, T // 3, T - 1])
+    ref = _run_forward(inp, dtype, c, path)
+    dev, tdt = _dev(inp, dtype)
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n, path=path)
+    guard = 4096
+    big = torch.full((plan.workspace_bytes + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    ws = big[guard:guard + plan.workspace_bytes]
+    assert ws.data_ptr() % 256 == 0
+    ws.fill_(0xFF)
+    ws[:256] = 0                                          # the status block is the one part that must be zero
+    plan.workspace = ws
+    M = torch.full((B, H, T), float("nan"), dtype=torch.float32, device="cuda")
+    O = torch.full((B, H, T, 64), float("nan"), dtype=tdt, device="cuda")
+    sel = torch.full((B, H, plan.u_max), -7, dtype=torch.int32, device="cuda")
+    for _ in range(2):                                    # the second call sees the first call's leftovers
+        plan.psattn_forward(dev["Q"], dev["K"], dev["V"], dev["lengths"], dev["sample_idx"], O, sel, M)
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() == 0
+    np.testing.assert_array_equal(O.float().cpu().numpy(), ref[0])
+    np.testing.assert_array_equal(sel.cpu().numpy(), ref[1])
+    np.testing.assert_array_equal(M.cpu().numpy(), ref[2])
+    assert bool((big[:guard] == 0xA5).all()) and bool((big[guard + plan.workspace_bytes:] == 0xA5).all())
+    plan.close()
+
+
+@pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_strided_bthd_layout(path):
     """Q, K, V, O stored [B][T][H][d] (projection output order) through the stride fields."""
     B, H, T, c, d = 2, 4, 160, 5.0, 64

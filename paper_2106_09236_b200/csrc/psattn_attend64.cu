@@ -33,12 +33,14 @@ __global__ void __launch_bounds__(kA64Threads, 1) k_attend64(Geom g, Attend64Arg
         if (tid == 0) atomicOr(g.status, kStatusWaitExpired);
         return;
     }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // programmatic dependent launch, see pdl_enter
     if (warp == 0) tmem_alloc(tmem_slot_p, kA64TmemCols);
     if (tid == 32) { tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_p;
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // nothing above touches global data
 
     Attend64Job j;
     j.b = unit / g.H; j.h = unit % g.H; j.L = seq_len(g, j.b);
@@ -143,7 +145,8 @@ cudaError_t launch_attend64(const Geom &g, const void *Q, const void *K, const v
         attr_set = true;
     }
     dim3 grid((unsigned)n_splits, (unsigned)(g.B * g.H));
-    k_attend64<<<grid, kA64Threads, kA64Bytes, st>>>(g, a, (const __nv_bfloat16 *)Q, tmK, tmV);
+    cudaError_t le = launch_pdl(k_attend64, grid, dim3(kA64Threads), kA64Bytes, st, g, a, (const __nv_bfloat16 *)Q, tmK, tmV);
+    if (le != cudaSuccess) { note_launch(); return le; }
     note_launch();
     return cudaGetLastError();
 }

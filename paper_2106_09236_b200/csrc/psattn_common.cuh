@@ -27,6 +27,15 @@ struct Geom {
     unsigned *status;                     // device status word
 };
 
+// Programmatic dependent launch, for kernels that are launched with launch_pdl (psattn_launch.h): lets the
+// next kernel of the stream be scheduled already, then waits until the previous kernel of the stream has
+// completed and its writes are visible.  Must run before the first access to global memory; both
+// instructions do nothing in a launch without the programmatic attribute.
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 __device__ __forceinline__ int seq_len(const Geom &g, int b) {
     if (!g.lengths) return g.T;
     int L = g.lengths[b];

@@ -11,6 +11,24 @@ constexpr int kSelectSmemKeys = 8192; // keys kept in shared memory by the selec
 constexpr int kSmCount = 148;         // SMs of a B200
 constexpr int kSplitKeys = 1024;      // keys per split of the SIMT attention kernel
 
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the
+// stream drains.  Only for kernels that call pdl_enter() before their first global-memory access.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args &&...args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Every kernel launch of the library is counted (process-wide).
 void note_launch(int n = 1);
 unsigned long long launches_so_far();

@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_measure_stream(Geom g, in
     const int tid = threadIdx.x;
     const int unit = blockIdx.x / q_slices, slice = blockIdx.x % q_slices;
     const int b = unit / g.H, h = unit % g.H;
+    pdl_enter();
     const int L = seq_len(g, b);
     const int U = min(g.U_tab[L], g.idx_cols);
     // slices in whole staged blocks so that every CTA but the last works on full blocks
@@ -172,10 +173,10 @@ cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const
         if (e != cudaSuccess) return e;
         attr_smem = smem;
     }
-    k_measure_stream<<<(unsigned)(units * slices), kStreamThreads, smem, st>>>(
-        g, slices, (uint32_t)stage_bytes, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, sidx, M);
+    cudaError_t e = launch_pdl(k_measure_stream, dim3((unsigned)(units * slices)), dim3(kStreamThreads), smem, st, g, slices,
+                               (uint32_t)stage_bytes, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, sidx, M);
     note_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace psattn

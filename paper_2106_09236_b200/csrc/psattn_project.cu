@@ -8,8 +8,8 @@
 // tcgen05.mma (M = 128, N = 192, K = 16) into one of two TMEM accumulators, warps 2-5 drain the other
 // accumulator: TMEM -> registers -> bf16 -> a swizzled staging tile -> whole 128-byte rows at (b, h, t).  The mainloop of tile i + 1 runs
 // under the drain of tile i.  Tiles that lie wholly beyond a sequence's length are skipped; rows beyond it
-// are not written.  For the V blocks the drain also reduces its 128 rows (as rounded to bf16) to one column
-// sum per block, in a fixed order, from which mean(V) - the fill value of step (e) - follows without
+// are not written.  For the V blocks every drain warp also adds up the columns of its 32 rows (as rounded to
+// bf16, read back from the staging tile), in a fixed order, from which mean(V) - the fill value of step (e) - follows without
 // another pass over V.
 // fp32 (and layouts without a tensor map): one thread per output element, fp32 FMA.
 #include "psattn_launch.h"
@@ -23,8 +23,7 @@ constexpr int kPjM = 128, kPjN = 192, kPjK = 64, kPjStages = 5;
 constexpr int kPjAccCols = 256;                                // TMEM columns reserved per accumulator
 constexpr uint32_t kPjBytesA = kPjM * kPjK * 2, kPjBytesB = kPjN * kPjK * 2, kPjStage = kPjBytesA + kPjBytesB;
 constexpr uint32_t kPjOffBar = kPjStages * kPjStage;           // mbarriers, TMEM slot, abort flag
-constexpr uint32_t kPjOffRed = kPjOffBar + 128;                // [4 warps][64] column-sum staging
-constexpr uint32_t kPjOffStage = kPjOffRed + 4 * 64 * 4;       // [4 warps][32 rows][128 B] output staging (swizzled)
+constexpr uint32_t kPjOffStage = kPjOffBar + 128;              // [4 warps][32 rows][128 B] output staging (swizzled)
 constexpr uint32_t kPjSmem = kPjOffStage + 4 * 4096;
 constexpr int kPjThreads = 192;
 
@@ -45,7 +44,7 @@ struct ProjArgs {
     long long qs[3], ks[3], vs[3];                // element strides (b, h, t) of the three outputs
     __nv_bfloat16 *Q, *K, *V;
     const int *lengths;
-    float *vpart;                                 // [B][tiles_per_seq][H][64] column sums of V per tile, or null
+    float *vpart;                                 // [B][tiles_per_seq][4][H][64] column sums of V per 32 rows, or null
     unsigned *status;
 };
 
@@ -66,7 +65,6 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
     uint64_t *acc_full = empty + kPjStages, *acc_empty = acc_full + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
-    float *red = reinterpret_cast<float *>(smem + kPjOffRed);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if ((smem_u32(smem) & 1023u) != 0u) {                      // swizzled tiles need a 1024-byte base
         if (tid == 0) atomicOr(a.status, kStatusWaitExpired);
@@ -140,7 +138,7 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
         }
     } else {
         // ---- drain: warp w reads TMEM lanes 32 (w % 4) .. + 31; thread = one token row ----
-        const int quarter = warp & 3, row = quarter * 32 + lane;
+        const int quarter = warp & 3;
         const int ew = warp - 2;                               // 0..3: slot in the staging buffers
         uint4 *stage = reinterpret_cast<uint4 *>(smem + kPjOffStage + ew * 4096);
         uint32_t tc = 0;
@@ -165,8 +163,6 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
                 break;
             }
             tc_fence_after();
-            const int t = tt * kPjM + row;
-            const bool valid = t < L;
             const int n_cc = min(kPjN / 64, 3 * a.H - n * (kPjN / 64));   // 64-column blocks of this tile
             const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kPjAccCols;
             uint32_t ra[64], rb[64];                           // two blocks in flight: the next one loads while
@@ -196,38 +192,27 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
                     const uint4 val = stage[rr * 8 + (c ^ (rr & 7))];
                     if (tr < L) reinterpret_cast<uint4 *>(base + (long long)tr * st[2])[c] = val;
                 }
-                __syncwarp();
                 if (role == 2 && a.vpart != nullptr) {
-                    // column sums of this block over the tile's valid rows, from the values as stored (bf16)
-                    float v[64];
+                    // column sums of this block over the warp's valid rows, from the values as stored (bf16):
+                    // lane l adds up word l (columns 2 l and 2 l + 1) of every row of the staging tile
+                    const int n_valid = min(32, max(0, L - (tt * kPjM + quarter * 32)));
+                    const uint32_t *words = reinterpret_cast<const uint32_t *>(stage);
+                    uint32_t wv[32];                           // all loads first: nothing else hides their latency here
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        v[2 * j] = valid ? __uint_as_float(pk[j] << 16) : 0.f;
-                        v[2 * j + 1] = valid ? __uint_as_float(pk[j] & 0xffff0000u) : 0.f;
-                    }
-                    // transposing butterfly: after the step with offset o a lane keeps half of its columns;
-                    // at the end lane l holds the sums of columns 2 l and 2 l + 1 over the warp's 32 rows
+                    for (int rr = 0; rr < 32; ++rr)
+                        wv[rr] = rr < n_valid ? words[rr * 32 + ((((lane >> 2) ^ (rr & 7)) << 2) | (lane & 3))] : 0u;
+                    float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int o = 16, cnt = 32; o >= 1; o >>= 1, cnt >>= 1) {
-                        const bool up = (lane & o) != 0;
-#pragma unroll
-                        for (int i = 0; i < cnt; ++i) {
-                            const float send = up ? v[i] : v[i + cnt];
-                            const float keep = up ? v[i + cnt] : v[i];
-                            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-                        }
+                    for (int rr = 0; rr < 32; ++rr) {          // four independent chains, combined in a fixed order
+                        e0[rr & 3] += __uint_as_float(wv[rr] << 16);
+                        e1[rr & 3] += __uint_as_float(wv[rr] & 0xffff0000u);
                     }
-                    red[ew * 64 + 2 * lane] = v[0];
-                    red[ew * 64 + 2 * lane + 1] = v[1];
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    const int et = tid - 64;                   // 0..127 within the drain warps
-                    if (et < 64) {
-                        // rows 0-31 are drained by warp 4 (slot 2), 32-63 by warp 5, 64-95 by warp 2, 96-127 by warp 3
-                        const float sum = ((red[2 * 64 + et] + red[3 * 64 + et]) + red[0 * 64 + et]) + red[1 * 64 + et];
-                        a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + et] = sum;
-                    }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const float s0 = (e0[0] + e0[1]) + (e0[2] + e0[3]), s1 = (e1[0] + e1[1]) + (e1[2] + e1[3]);
+                    float2 *dst = reinterpret_cast<float2 *>(
+                        a.vpart + ((((long long)b * a.tiles_per_seq + tt) * 4 + quarter) * a.H + h) * 64);
+                    dst[lane] = make_float2(s0, s1);
                 }
+                __syncwarp();
             };
 #pragma unroll
             for (int cc = 0; cc < kPjN / 64; cc += 2) {
@@ -262,7 +247,8 @@ __global__ void __launch_bounds__(64) k_project_vbar(ProjArgs a, float *__restri
     asm volatile("griddepcontrol.wait;" ::: "memory");        // the per-tile sums of the kernel before
     const int L = proj_len(a, b);
     float s = 0.f;
-    for (int tt = 0; tt * kPjM < L; ++tt) s += a.vpart[(((long long)b * a.tiles_per_seq + tt) * a.H + h) * 64 + e];
+    for (int tt = 0; tt * kPjM < L; ++tt)
+        for (int q = 0; q < 4; ++q) s += a.vpart[((((long long)b * a.tiles_per_seq + tt) * 4 + q) * a.H + h) * 64 + e];
     vbar[(long long)unit * 64 + e] = L > 0 ? s / (float)L : 0.f;
 }
 
@@ -315,7 +301,7 @@ static EncodeTiledFnP proj_encode_fn() {
     return fn;
 }
 
-size_t project_vpart_floats(int B, int H, int T) { return (size_t)B * ((T + kPjM - 1) / kPjM) * H * 64; }
+size_t project_vpart_floats(int B, int H, int T) { return (size_t)B * ((T + kPjM - 1) / kPjM) * 4 * H * 64; }
 
 // dtype 0 = bf16, 1 = fp32.  X [B][T][dx], Wt [3][H*64][dx], outputs with g.qs / g.ks / g.vs strides.
 // vbar (optional) fp32 [B][H][64]; vpart = scratch of project_vpart_floats() floats (needed with vbar on the

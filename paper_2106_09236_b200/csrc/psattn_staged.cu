@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(256) k_colsum(Geom g, const DT *__restrict__ V
     __shared__ float red[32][kD + 1];
     const int unit = blockIdx.x, chunk = blockIdx.y;
     const int b = unit / g.H, h = unit % g.H;
+    pdl_enter();
     const int L = seq_len(g, b);
     const int sub = threadIdx.x & 7, r0 = threadIdx.x >> 3;
     const int lo = chunk * kColsumRows, hi = min(L, lo + kColsumRows);
@@ -130,6 +131,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *
     __shared__ SelectScratch scratch;
     const int unit = blockIdx.x;
     const int b = unit / g.H;
+    pdl_enter();
     const int L = seq_len(g, b);
     const int u = min(min(g.u_tab[L], g.u_max), L);
     const float *Mu = M + (long long)unit * g.T;
@@ -262,6 +264,7 @@ __global__ void __launch_bounds__(256) k_attend_combine(Geom g, const int *__res
                                                         long long out_row_stride,
                                                         int out_by_position, float *__restrict__ vbar) {
     const int n_slots = n_rows + (vbar ? 1 : 0);           // slot n_rows (if any) is the all-ones row
+    pdl_enter();
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long rowid = t / kD;
     const int c = (int)(t % kD);
@@ -314,6 +317,7 @@ __global__ void __launch_bounds__(256) k_fill(Geom g, const DT *__restrict__ V,
     __shared__ unsigned char chosen[kFillRows];
     const int unit = blockIdx.x;
     const int b = unit / g.H, h = unit % g.H;
+    pdl_enter();
     const int L = seq_len(g, b);
     const int lo = blockIdx.y * kFillRows;
     for (int t = threadIdx.x; t < kFillRows; t += blockDim.x) chosen[t] = 0;
@@ -365,8 +369,10 @@ cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, 
                           cudaStream_t st) {
     if (g.B * g.H == 0 || n_chunks == 0) return cudaSuccess;
     dim3 grid((unsigned)(g.B * g.H), (unsigned)n_chunks);
-    if (dtype == 0) k_colsum<__nv_bfloat16><<<grid, 256, 0, st>>>(g, (const __nv_bfloat16 *)V, part, n_chunks);
-    else k_colsum<float><<<grid, 256, 0, st>>>(g, (const float *)V, part, n_chunks);
+    cudaError_t e;
+    if (dtype == 0) e = launch_pdl(k_colsum<__nv_bfloat16>, grid, dim3(256), 0, st, g, (const __nv_bfloat16 *)V, part, n_chunks);
+    else e = launch_pdl(k_colsum<float>, grid, dim3(256), 0, st, g, (const float *)V, part, n_chunks);
+    if (e != cudaSuccess) return e;
     note_launch();
     return cudaGetLastError();
 }
@@ -374,7 +380,9 @@ cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, 
 cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,
                           float *vbar, cudaStream_t st) {
     if (g.B * g.H == 0) return cudaSuccess;
-    k_select<<<(unsigned)(g.B * g.H), kSelectThreads, 0, st>>>(g, M, sel, vpart, n_chunks, vbar); note_launch();
+    cudaError_t e = launch_pdl(k_select, dim3((unsigned)(g.B * g.H)), dim3(kSelectThreads), 0, st, g, M, sel, vpart, n_chunks, vbar);
+    note_launch();
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
@@ -416,28 +424,30 @@ cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows,
     const long long threads = (long long)g.B * g.H * (n_rows + (vbar ? 1 : 0)) * kD;
     if (threads == 0) return cudaSuccess;
     const unsigned blocks = (unsigned)((threads + 255) / 256);
+    cudaError_t e;
     if (out_is_bf16)
-        k_attend_combine<__nv_bfloat16><<<blocks, 256, 0, st>>>(g, rows, n_rows, rows_stride, n_splits, part_ml,
-                                                                 part_acc, (__nv_bfloat16 *)out, out_unit_stride,
-                                                                 out_row_stride, out_by_position, vbar);
+        e = launch_pdl(k_attend_combine<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, g, rows, n_rows, rows_stride,
+                       n_splits, part_ml, part_acc, (__nv_bfloat16 *)out, out_unit_stride, out_row_stride,
+                       out_by_position, vbar);
     else
-        k_attend_combine<float><<<blocks, 256, 0, st>>>(g, rows, n_rows, rows_stride, n_splits, part_ml, part_acc,
-                                                        (float *)out, out_unit_stride, out_row_stride,
-                                                        out_by_position, vbar);
+        e = launch_pdl(k_attend_combine<float>, dim3(blocks), dim3(256), 0, st, g, rows, n_rows, rows_stride, n_splits,
+                       part_ml, part_acc, (float *)out, out_unit_stride, out_row_stride, out_by_position, vbar);
     note_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
                         void *O, int own_v, cudaStream_t st) {
     if (g.B * g.H == 0 || g.T == 0) return cudaSuccess;
     dim3 grid((unsigned)(g.B * g.H), (unsigned)((g.T + kFillRows - 1) / kFillRows));
+    cudaError_t e;
     if (dtype == 0)
-        k_fill<__nv_bfloat16><<<grid, 256, 0, st>>>(g, (const __nv_bfloat16 *)V, sel, vbar, (__nv_bfloat16 *)O, own_v);
+        e = launch_pdl(k_fill<__nv_bfloat16>, grid, dim3(256), 0, st, g, (const __nv_bfloat16 *)V, sel, vbar,
+                       (__nv_bfloat16 *)O, own_v);
     else
-        k_fill<float><<<grid, 256, 0, st>>>(g, (const float *)V, sel, vbar, (float *)O, own_v);
+        e = launch_pdl(k_fill<float>, grid, dim3(256), 0, st, g, (const float *)V, sel, vbar, (float *)O, own_v);
     note_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace psattn

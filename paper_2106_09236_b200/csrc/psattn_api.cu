@@ -345,7 +345,7 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
     Geom g = make_geom(plan, lengths, workspace);
     if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && !d.idx_shared) {
         cudaError_t e = launch_forward_fused(g, plan->U_max, d.fill_mode == PSATTN_FILL_OWN_V, Q, K, V, sample_idx, O,
-                                             sel_idx, M_out, st);
+                                             sel_idx, M_out, nullptr, st);
         if (e == cudaSuccess) return PSATTN_OK;
         if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
         if (d.path == PSATTN_PATH_FUSED) return PSATTN_ERR_UNSUPPORTED;
@@ -375,6 +375,13 @@ extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && d.B * d.H >= kSmCount / 2) {
+        // one kernel for steps (d)+(e), one CTA per unit: where the units cover at least half of the SMs
+        cudaError_t e = launch_forward_fused(g, plan->U_max, d.fill_mode == PSATTN_FILL_OWN_V, Q, K, V, nullptr, O,
+                                             nullptr, nullptr, sel_idx_in, st);
+        if (e == cudaSuccess) return PSATTN_OK;
+        if (e != cudaErrorNotSupported) return cuda_fail(plan, e);
+    }
     if (vbar_from_attention(plan, g, K, V))
         return run_attend_and_fill(plan, g, Q, K, V, sel_idx_in, O, workspace, st, false);
     // mean(V) by a column-sum pass (the select kernel, run without keys, only finishes the mean)

@@ -9,6 +9,8 @@
 //      tensor cores while V streams through, so V is read from HBM once        (Eq. 7-8; Sec. 3.1)
 //   4. mean(V) (or the query's own value row) is written to every other valid row of O, zeros
 //      to padded rows                                                         (Eq. 12)
+// With a given index set (the reuse of one layer's selection by the following layers, Sec. 4.4) steps
+// 1 and 2 are skipped and the kernel is steps (d)+(e) in one launch.
 // HBM traffic is the algorithmic minimum: Q, K, V read once (K a second time out of L2), O
 // written once.  M~ never leaves the SM unless the caller asks for it.
 #include "psattn_attend64.cuh"
@@ -28,6 +30,7 @@ struct FusedArgs {
     int pos_t, pos_h, pos_b;             // TMA coordinate slots (same for the three maps)
     int own_v;                           // fill with the query's own value row instead of mean(V)
     int by_length;                       // CTAs take the sequences in descending order of length
+    const int *sel_in;                   // non-null: a given index set [unit][u_max] replaces steps (a)-(c)
 };
 
 struct FusedPersist {                    // at smem + off_persist + 4 * T (after the M~ array)
@@ -84,10 +87,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     const int L = seq_len(g, b);
     const int U = min(g.U_tab[L], g.idx_cols);
     const int u = min(min(g.u_tab[L], g.u_max), L);
+    const bool given = a.sel_in != nullptr;                    // steps (d)+(e) only, for a given index set
     if (tid == 32) {
         mbar_init(&P.bar, 1);
         fence_barrier_init();
-        if (L > 0) measure_issue_keys(smem, &P.bar, &tmKrows, L, b, h, a.pos_t, a.pos_h);
+        if (L > 0 && !given) measure_issue_keys(smem, &P.bar, &tmKrows, L, b, h, a.pos_t, a.pos_h);
         tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
     }
     for (int i = tid; i < g.T; i += kFusedThreads) { chosen[i] = 0; if (i >= L) M_s[i] = 0.f; }
@@ -98,30 +102,39 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
 
     // ---- steps (a)+(b) ------------------------------------------------------------------------
     bool ok = true;
-    if (L > 0)
+    if (L > 0 && !given)
         ok = measure_resident<kFusedThreads>(smem, &P.bar, 0u, a.k_bytes, a.stage_bytes, g, unit, b, h, L, U, 0, L, Q,
                                              sidx, M_s);
     __syncthreads();
-    if (M_out != nullptr)
+    if (M_out != nullptr && !given)
         for (int i = tid; i < g.T; i += kFusedThreads) M_out[(long long)unit * g.T + i] = M_s[i];
 
     // The attention phase reuses the shared memory of the measure phase, which is free now; its first
     // K/V tiles depend only on the unit, so their copies start before the selection and land behind it.
     Attend64Job j;
     j.b = b; j.h = h; j.L = L; j.lo = 0; j.hi = L;
-    j.rows = P.sel; j.n_rows = u;
+    const int n_rows = given ? g.u_max : u;                    // a given list is taken at its full width
+    j.rows = P.sel; j.n_rows = n_rows;
     j.pos_t = a.pos_t; j.pos_h = a.pos_h; j.pos_b = a.pos_b;
     j.ctrl_warp = 0; j.wg_warp0 = 4;
-    j.sum_row = a.own_v ? -1 : u;
+    j.sum_row = a.own_v ? -1 : n_rows;
     j.started = 1;
     if (ok && L > 0 && tid == 0) attend64_start(smem, j, &tmK, &tmV);
 
     // ---- step (c) -----------------------------------------------------------------------------
-    block_select([&](int i) { return float_key(M_s[i]); }, L, u, kA64MaxRows, P.sel, P.select);
-    for (int r = tid; r < g.u_max; r += kFusedThreads) {
-        const int i = r < kA64MaxRows ? P.sel[r] : -1;
-        sel_out[(long long)unit * g.u_max + r] = i;
-        if (i >= 0) chosen[i] = 1;
+    if (!given) {
+        block_select([&](int i) { return float_key(M_s[i]); }, L, u, kA64MaxRows, P.sel, P.select);
+        for (int r = tid; r < g.u_max; r += kFusedThreads) {
+            const int i = r < kA64MaxRows ? P.sel[r] : -1;
+            sel_out[(long long)unit * g.u_max + r] = i;
+            if (i >= 0) chosen[i] = 1;
+        }
+    } else {
+        for (int r = tid; r < kA64MaxRows; r += kFusedThreads) {
+            const int i = r < g.u_max ? a.sel_in[(long long)unit * g.u_max + r] : -1;
+            P.sel[r] = (i >= 0 && i < L) ? i : -1;              // entries outside the sequence are ignored
+            if (i >= 0 && i < L) chosen[i] = 1;
+        }
     }
     __syncthreads();
 
@@ -132,13 +145,15 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
         if (ok && warp >= 4 && warp < 8 && lane < 16) {
             const int r = 16 * (warp - 4) + lane;
             const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            if (r < u) {
+            if (r < n_rows) {
                 const int i = P.sel[r];
+                if (i >= 0) {
 #pragma unroll
-                for (int c = 0; c < kD; ++c) acc[c] *= inv;
-                __nv_bfloat16 *dst = O + unit_off(g.os, b, h) + (long long)i * g.os[2];
+                    for (int c = 0; c < kD; ++c) acc[c] *= inv;
+                    __nv_bfloat16 *dst = O + unit_off(g.os, b, h) + (long long)i * g.os[2];
 #pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) store8(dst, c8, acc + 8 * c8);
+                    for (int c8 = 0; c8 < 8; ++c8) store8(dst, c8, acc + 8 * c8);
+                }
             } else if (r == j.sum_row) {
 #pragma unroll
                 for (int c = 0; c < kD; ++c) P.vbar[c] = acc[c] * inv;     // l = number of valid keys
@@ -174,9 +189,10 @@ bool make_rows_map(CUtensorMap *map, const void *base, const Geom &g, const long
 // cudaErrorNotSupported when the shape does not fit this kernel (the caller runs the staged schedule):
 // keys + staging beyond shared memory, more than 63 selected rows or 64 samples, no tensor map.
 cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void *Q, const void *K, const void *V,
-                                 const int *sidx, void *O, int *sel, float *M_out, cudaStream_t st) {
+                                 const int *sidx, void *O, int *sel, float *M_out, const int *sel_in, cudaStream_t st) {
     if (g.B * g.H == 0) return cudaSuccess;
-    if (g.u_max > kA64MaxRows - 1 || U_max > kMeasureMaxU || U_max < 1) return cudaErrorNotSupported;
+    if (g.u_max > kA64MaxRows - 1) return cudaErrorNotSupported;
+    if (sel_in == nullptr && (U_max > kMeasureMaxU || U_max < 1)) return cudaErrorNotSupported;
     FusedArgs a;
     a.k_bytes = (uint32_t)measure_k_bytes(g.T);
     a.stage_bytes = (uint32_t)measure_stage_bytes(kFusedThreads, g.idx_cols);
@@ -194,6 +210,7 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
         if (p0[x] != p1[x] || p1[x] != p2[x]) return cudaErrorNotSupported;
     a.pos_t = p0[0]; a.pos_h = p0[1]; a.pos_b = p0[2];
     a.own_v = own_v;
+    a.sel_in = sel_in;
     // the ranking costs B comparisons per sequence in every CTA: only where a second wave exists and B is small
     a.by_length = g.lengths != nullptr && g.B * g.H > kSmCount && g.B <= 256;
     static size_t attr_smem = 0;

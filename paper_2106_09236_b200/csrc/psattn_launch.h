@@ -42,8 +42,9 @@ cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const vo
                                cudaStream_t st);
 // Steps (a)-(e) of every unit in one kernel (bf16, keys resident in shared memory).
 // cudaErrorNotSupported: shape outside the kernel's limits; run the staged schedule instead.
+// sel_in != nullptr: steps (d)+(e) only, for the given index set [unit][u_max] (sidx, sel, M_out unused).
 cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void *Q, const void *K, const void *V,
-                                 const int *sidx, void *O, int *sel, float *M_out, cudaStream_t st);
+                                 const int *sidx, void *O, int *sel, float *M_out, const int *sel_in, cudaStream_t st);
 // Streaming tensor-datapath form of steps (a)+(b) for bf16 inputs and any T_max (key rows gathered from L2
 // through shared-memory rings); cudaErrorNotSupported when U_max > 64.
 cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const void *K, const int *sidx, float *M,

@@ -425,6 +425,43 @@ def test_forward_with_given_selection(path):
     plan.close()
 
 
+@pytest.mark.parametrize("fill", ["mean_v", "own_v"])
+@pytest.mark.parametrize("T", [200, 1024])
+def test_forward_with_given_selection_one_kernel_form(T, fill):
+    """Enough units that steps (d)+(e) run as one kernel per unit; the list is unsorted, shorter than its
+    width for short sequences, and holds entries outside the sequence (ignored) in some units."""
+    B, H, c = 21, 4, 5.0
+    rng = np.random.default_rng(77 + T)
+    lengths = rng.integers(1, T + 1, size=B).astype(np.int32)
+    lengths[0], lengths[1] = T, 1
+    n = orc.count(c, T)
+    inp = _synth(B, H, T, 61, n, "bf16", lengths)
+    dev, tdt = _dev(inp, "bf16")
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n,
+                   fill_mode=ps.PSATTN_FILL_OWN_V if fill == "own_v" else ps.PSATTN_FILL_MEAN_V)
+    sel_in = np.full((B, H, plan.u_max), -1, dtype=np.int32)
+    for b in range(B):
+        for h in range(H):
+            k = min(plan.u_max, int(lengths[b]), orc.count(c, int(lengths[b])) + 3)
+            sel_in[b, h, :k] = rng.permutation(int(lengths[b]))[:k]           # unsorted
+    given = sel_in.copy()
+    given[2, 1, -1] = int(lengths[2]) + 5 if lengths[2] + 5 < 2 ** 30 else -1  # beyond the sequence: ignored
+    given[3, 0, -1] = -9
+    clean = given.copy()
+    clean[2, 1, -1] = -1
+    clean[3, 0, -1] = -1
+    O = torch.full((B, H, T, 64), float("nan"), dtype=tdt, device="cuda")
+    before = ps.psattn_launch_count()
+    plan.psattn_forward_with_selection(dev["Q"], dev["K"], dev["V"], dev["lengths"], torch.from_numpy(given).cuda(), O)
+    torch.cuda.synchronize()
+    assert ps.psattn_launch_count() - before == 1
+    assert plan.psattn_read_status() == 0
+    O_ref, _, _ = orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=c, sel_in=clean,
+                              fill=fill, nthreads=orc.max_threads())
+    parity.check_outputs(O.float().cpu().numpy(), O_ref, {}, inp, inp["lengths"], "bf16")
+    plan.close()
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
 def test_dense_comparator(dtype):
     B, H, T = 2, 2, 300

@@ -16,8 +16,12 @@
  *
  * Conventions common to every call
  *   - All functions return an int status (PSATTN_OK == 0); none throws, aborts or
- *     synchronises the device, except where stated.  All device work is enqueued on
- *     the caller's stream (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *     synchronises the device, except where stated.  All device work is ordered on
+ *     the caller's stream (a cudaStream_t passed as void*; NULL = the legacy default stream):
+ *     it is enqueued there, except that psattn_forward may run the part of step (e) that does
+ *     not depend on steps (a)-(c) on a stream owned by the plan, forked from and joined back
+ *     into the caller's stream with events inside the call (which a stream capture follows).
+ *     Calls on one plan must therefore be stream-ordered with each other.
  *   - "device" pointers must be device memory of the GPU that was current when the
  *     plan was created; "host" pointers are ordinary host memory.  The caller owns every
  *     buffer.  After psattn_plan_create the library allocates nothing (exception:

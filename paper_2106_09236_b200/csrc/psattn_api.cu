@@ -29,6 +29,9 @@ struct psattn_plan {
     cudaStream_t h_copy_stream;   // device-to-host copies of finished chunks run here
     cudaEvent_t h_ev[2];          // [0]: a chunk is finished; [1]: its results have been copied out
     int b_override;               // > 0: number of sequences of the current (chunked) call
+    // side stream of the staged schedule: the fill of step (e) runs there while steps (a)-(c) run on the caller's
+    cudaStream_t side_stream;
+    cudaEvent_t side_ev[2];       // [0]: fork (recorded on the caller's stream), [1]: join (recorded on the side stream)
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -158,6 +161,15 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     // per-tile column sums of V written by the projection kernel
     p->off_pvsum = off;  off = align_up(off + project_vpart_floats(d.B, d.H, d.T_max) * sizeof(float), 256);
     p->ws_bytes = off;
+    if (cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->side_ev[0], cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&p->side_ev[1], cudaEventDisableTiming) != cudaSuccess) {
+        if (p->side_ev[0]) cudaEventDestroy(p->side_ev[0]);
+        if (p->side_stream) cudaStreamDestroy(p->side_stream);
+        cudaFree(p->d_tables);
+        delete p;
+        return PSATTN_ERR_CUDA;
+    }
     *out = p;
     return PSATTN_OK;
 }
@@ -165,6 +177,7 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
 extern "C" int psattn_plan_destroy(psattn_plan_t *p) {
     if (!p) return PSATTN_ERR_NULL;
     cudaFree(p->d_tables);
+    cudaStreamDestroy(p->side_stream); cudaEventDestroy(p->side_ev[0]); cudaEventDestroy(p->side_ev[1]);
     if (p->host_io) {
         cudaFree(p->h_Q); cudaFree(p->h_K); cudaFree(p->h_V); cudaFree(p->h_O); cudaFree(p->h_ws);
         cudaFree(p->h_len); cudaFree(p->h_idx); cudaFree(p->h_sel);
@@ -353,11 +366,33 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
         return PSATTN_ERR_UNSUPPORTED;
     }
     float *M = M_out ? M_out : ws_at<float>(workspace, plan->off_M);
-    if ((rc = run_measure(plan, g, Q, K, sample_idx, M, st)) != PSATTN_OK) return rc;
     if (vbar_from_attention(plan, g, K, V)) {
-        PSATTN_CU(launch_select(g, M, sel_idx, nullptr, 0, nullptr, st));
-        return run_attend_and_fill(plan, g, Q, K, V, sel_idx, O, workspace, st, false);
+        // Steps (a)-(c) do not touch V or O, and they are bound by on-chip gathers, not by HBM: the fill of
+        // step (e) - column sums of V, mean(V), every valid row of O - runs beside them on the plan's side
+        // stream (forked and joined with events, so the call stays ordered on the caller's stream and can be
+        // captured in a graph); step (d) then overwrites the selected rows.
+        float *vbar = ws_at<float>(workspace, plan->off_vbar);
+        PSATTN_CU(cudaEventRecord(plan->side_ev[0], st));
+        PSATTN_CU(cudaStreamWaitEvent(plan->side_stream, plan->side_ev[0], 0));
+        cudaError_t se = cudaSuccess;
+        if (d.fill_mode == PSATTN_FILL_MEAN_V) {
+            se = launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, plan->side_stream);
+            if (se == cudaSuccess)
+                se = launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, vbar,
+                                   plan->side_stream);
+        }
+        if (se == cudaSuccess)
+            se = launch_fill(d.dtype, g, V, nullptr, vbar, O, d.fill_mode == PSATTN_FILL_OWN_V, plan->side_stream);
+        // always join, whatever happened on either side
+        cudaError_t je = cudaEventRecord(plan->side_ev[1], plan->side_stream);
+        rc = run_measure(plan, g, Q, K, sample_idx, M, st);
+        cudaError_t le = rc == PSATTN_OK ? launch_select(g, M, sel_idx, nullptr, 0, nullptr, st) : cudaSuccess;
+        if (je == cudaSuccess) je = cudaStreamWaitEvent(st, plan->side_ev[1], 0);
+        if (rc != PSATTN_OK) return rc;
+        PSATTN_CU(se); PSATTN_CU(je); PSATTN_CU(le);
+        return run_attend(plan, g, Q, K, V, sel_idx, plan->u_max, plan->u_max, O, 0, 0, 1, 0, workspace, st);
     }
+    if ((rc = run_measure(plan, g, Q, K, sample_idx, M, st)) != PSATTN_OK) return rc;
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
     PSATTN_CU(launch_select(g, M, sel_idx, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks,
                             ws_at<float>(workspace, plan->off_vbar), st));

@@ -322,10 +322,11 @@ __global__ void __launch_bounds__(256) k_fill(Geom g, const DT *__restrict__ V,
     const int lo = blockIdx.y * kFillRows;
     for (int t = threadIdx.x; t < kFillRows; t += blockDim.x) chosen[t] = 0;
     __syncthreads();
-    for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) {
-        const int i = sel[(long long)unit * g.u_max + r];
-        if (i >= lo && i < lo + kFillRows && i < L) chosen[i - lo] = 1;
-    }
+    if (sel != nullptr)                                    // no list: every valid row is filled
+        for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) {
+            const int i = sel[(long long)unit * g.u_max + r];
+            if (i >= lo && i < lo + kFillRows && i < L) chosen[i - lo] = 1;
+        }
     __syncthreads();
     const int sub = threadIdx.x & 7, r0 = threadIdx.x >> 3;
     float mean8[8], zero8[8];

@@ -240,16 +240,27 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
     if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
-// mean(V) of every unit from the per-tile column sums, in tile order.
-__global__ void __launch_bounds__(64) k_project_vbar(ProjArgs a, float *__restrict__ vbar) {
-    const int unit = blockIdx.x, b = unit / a.H, h = unit % a.H, e = threadIdx.x;
+// mean(V) of every unit from the partial column sums: eight groups of 64 threads take every eighth partial
+// (in order), the eight group sums are then added in order.
+__global__ void __launch_bounds__(512) k_project_vbar(ProjArgs a, float *__restrict__ vbar) {
+    __shared__ float red[8][64];
+    const int unit = blockIdx.x, b = unit / a.H, h = unit % a.H, e = threadIdx.x & 63, grp = threadIdx.x >> 6;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    asm volatile("griddepcontrol.wait;" ::: "memory");        // the per-tile sums of the kernel before
+    asm volatile("griddepcontrol.wait;" ::: "memory");        // the partial sums of the kernel before
     const int L = proj_len(a, b);
+    const int n_part = ((L + kPjM - 1) / kPjM) * 4;            // one partial per 32 rows of every tile in use
+    const float *base = a.vpart + ((long long)b * a.tiles_per_seq * 4 * a.H + h) * 64 + e;
     float s = 0.f;
-    for (int tt = 0; tt * kPjM < L; ++tt)
-        for (int q = 0; q < 4; ++q) s += a.vpart[((((long long)b * a.tiles_per_seq + tt) * 4 + q) * a.H + h) * 64 + e];
-    vbar[(long long)unit * 64 + e] = L > 0 ? s / (float)L : 0.f;
+#pragma unroll 4
+    for (int p = grp; p < n_part; p += 8) s += base[(long long)p * a.H * 64];
+    red[grp][e] = s;
+    __syncthreads();
+    if (grp == 0) {
+        float t = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) t += red[q][e];
+        vbar[(long long)unit * 64 + e] = L > 0 ? t / (float)L : 0.f;
+    }
 }
 
 // Any element type and layout: one thread per output element (64 threads = one head block of one token).
@@ -357,7 +368,7 @@ cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx,
             if (e == cudaSuccess) e = cudaGetLastError();
             if (e != cudaSuccess || vbar == nullptr) return e;
             cfg.gridDim = dim3((unsigned)(g.B * g.H));
-            cfg.blockDim = dim3(64);
+            cfg.blockDim = dim3(512);
             cfg.dynamicSmemBytes = 0;
             e = cudaLaunchKernelEx(&cfg, k_project_vbar, a, vbar);
             note_launch();

@@ -21,7 +21,7 @@ struct psattn_plan {
     int *d_tables;                // device: u_tab[T+1] then U_tab[T+1]
     int last_cuda_error;
     // workspace layout (byte offsets)
-    size_t off_status, off_M, off_vpart, off_vbar, off_ml, off_acc, off_sel, off_pvsum, ws_bytes;
+    size_t off_status, off_M, off_vpart, off_vbar, off_ml, off_acc, off_sel, off_pvsum, off_cand, ws_bytes;
     // host-io staging (psattn_plan_enable_host_io)
     bool host_io;
     void *h_Q, *h_K, *h_V, *h_O, *h_ws;
@@ -160,6 +160,8 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     p->off_sel = off;    off = align_up(off + units * u_max * sizeof(int), 256);
     // per-tile column sums of V written by the projection kernel
     p->off_pvsum = off;  off = align_up(off + project_vpart_floats(d.B, d.H, d.T_max) * sizeof(float), 256);
+    // candidates of the two-kernel selection
+    p->off_cand = off;   off = align_up(off + select_cand_ints((int)units, u_max) * sizeof(int), 256);
     p->ws_bytes = off;
     if (cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&p->side_ev[0], cudaEventDisableTiming) != cudaSuccess ||
@@ -379,14 +381,14 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
             se = launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, plan->side_stream);
             if (se == cudaSuccess)
                 se = launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, vbar,
-                                   plan->side_stream);
+                                   nullptr, plan->side_stream);
         }
         if (se == cudaSuccess)
             se = launch_fill(d.dtype, g, V, nullptr, vbar, O, d.fill_mode == PSATTN_FILL_OWN_V, plan->side_stream);
         // always join, whatever happened on either side
         cudaError_t je = cudaEventRecord(plan->side_ev[1], plan->side_stream);
         rc = run_measure(plan, g, Q, K, sample_idx, M, st);
-        cudaError_t le = rc == PSATTN_OK ? launch_select(g, M, sel_idx, nullptr, 0, nullptr, st) : cudaSuccess;
+        cudaError_t le = rc == PSATTN_OK ? launch_select(g, M, sel_idx, nullptr, 0, nullptr, ws_at<int>(workspace, plan->off_cand), st) : cudaSuccess;
         if (je == cudaSuccess) je = cudaStreamWaitEvent(st, plan->side_ev[1], 0);
         if (rc != PSATTN_OK) return rc;
         PSATTN_CU(se); PSATTN_CU(je); PSATTN_CU(le);
@@ -395,7 +397,7 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
     if ((rc = run_measure(plan, g, Q, K, sample_idx, M, st)) != PSATTN_OK) return rc;
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
     PSATTN_CU(launch_select(g, M, sel_idx, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks,
-                            ws_at<float>(workspace, plan->off_vbar), st));
+                            ws_at<float>(workspace, plan->off_vbar), nullptr, st));
     return run_attend_and_fill(plan, g, Q, K, V, sel_idx, O, workspace, st, true);
 }
 
@@ -422,7 +424,7 @@ extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q,
     // mean(V) by a column-sum pass (the select kernel, run without keys, only finishes the mean)
     PSATTN_CU(launch_colsum(d.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
     PSATTN_CU(launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart),
-                            plan->n_chunks, ws_at<float>(workspace, plan->off_vbar), st));
+                            plan->n_chunks, ws_at<float>(workspace, plan->off_vbar), nullptr, st));
     return run_attend_and_fill(plan, g, Q, K, V, sel_idx_in, O, workspace, st, true);
 }
 
@@ -473,7 +475,8 @@ extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t 
     int rc = check_ws(plan, workspace, workspace_bytes);
     if (rc) return rc;
     Geom g = make_geom(plan, lengths, workspace);
-    PSATTN_CU(launch_select(g, M, sel_idx, nullptr, 0, nullptr, static_cast<cudaStream_t>(stream)));
+    PSATTN_CU(launch_select(g, M, sel_idx, nullptr, 0, nullptr, ws_at<int>(workspace, plan->off_cand),
+                            static_cast<cudaStream_t>(stream)));
     return PSATTN_OK;
 }
 
@@ -486,7 +489,7 @@ extern "C" int psattn_mean_v(psattn_plan_t *plan, const void *V, const int32_t *
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     Geom g = make_geom(plan, lengths, workspace);
     PSATTN_CU(launch_colsum(plan->desc.dtype, g, V, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, st));
-    PSATTN_CU(launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, vbar, st));
+    PSATTN_CU(launch_select(g, nullptr, nullptr, ws_at<float>(workspace, plan->off_vpart), plan->n_chunks, vbar, nullptr, st));
     return PSATTN_OK;
 }
 

@@ -56,8 +56,11 @@ cudaError_t launch_measure_shared(const Geom &g, int U_max, const void *Q, const
                                   cudaStream_t st);
 cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, int n_chunks,
                           cudaStream_t st);
+// cand (optional): scratch of select_cand_ints(units, u_max) ints; with it, few units of long sequences are
+// selected in two kernels (ranges of positions first, then their candidates).
+size_t select_cand_ints(int units, int u_max);
 cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,
-                          float *vbar, cudaStream_t st);
+                          float *vbar, int *cand, cudaStream_t st);
 // rows == nullptr: the row list is the identity (row r is position r).
 // out_by_position: write the finished row at its position in O (element type of the inputs,
 // strides g.os); otherwise at slot r of `out` with the given unit / row strides.

@@ -155,6 +155,62 @@ __global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *
 }
 
 // ---------------------------------------------------------------------------------------
+// Step (c) for few units with long sequences, in two kernels: every unit is cut into `slices` ranges of
+// `width` positions; one block per (unit, range) finds the top-u of its range (an element of the unit's
+// top-u is also in the top-u of its own range); one small block per unit then picks the top-u among the
+// slices * u candidates, which sit in position order, so that the tie rule (equal values: lower position
+// first) carries over.  Four times as many SMs work on the long scan, and each block's scan is short.
+// ---------------------------------------------------------------------------------------
+constexpr int kSelectMaxSlices = 8;
+
+__global__ void __launch_bounds__(kSelectThreads) k_select_slice(Geom g, const float *__restrict__ M, int slices,
+                                                                 int width, int *__restrict__ cand) {
+    __shared__ SelectScratch scratch;
+    __shared__ unsigned keys[kSelectSmemKeys];
+    const int unit = blockIdx.x / slices, sl = blockIdx.x % slices;
+    const int b = unit / g.H;
+    pdl_enter();
+    const int L = seq_len(g, b);
+    const int u = min(min(g.u_tab[L], g.u_max), L);
+    const int lo = sl * width, n = max(0, min(L - lo, width));
+    const float *Mu = M + (long long)unit * g.T + lo;
+    int *out = cand + ((long long)unit * slices + sl) * g.u_max;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = float_key(Mu[i]);
+    __syncthreads();
+    block_select([&](int i) { return keys[i]; }, n, min(u, n), g.u_max, out, scratch);
+    for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) {       // positions within the range -> positions of the unit
+        const int p = out[r];
+        if (p >= 0) out[r] = p + lo;
+    }
+}
+
+__global__ void __launch_bounds__(256) k_select_merge(Geom g, const float *__restrict__ M, int slices,
+                                                      const int *__restrict__ cand, int *__restrict__ sel) {
+    __shared__ SelectScratch scratch;
+    __shared__ unsigned ckey[kSelectMaxSlices * 64];
+    __shared__ int cidx[kSelectMaxSlices * 64];
+    const int unit = blockIdx.x;
+    const int b = unit / g.H;
+    pdl_enter();
+    const int L = seq_len(g, b);
+    const int u = min(min(g.u_tab[L], g.u_max), L);
+    const int n = slices * g.u_max;                            // candidate slots, -1 padded per range
+    const float *Mu = M + (long long)unit * g.T;
+    for (int p = threadIdx.x; p < n; p += blockDim.x) {
+        const int i = cand[(long long)unit * n + p];
+        cidx[p] = i;
+        ckey[p] = i >= 0 ? float_key(Mu[i]) : 0u;              // 0 lies below the key of every float
+    }
+    __syncthreads();
+    int *out = sel + (long long)unit * g.u_max;
+    block_select([&](int p) { return ckey[p]; }, n, u, g.u_max, out, scratch);
+    for (int r = threadIdx.x; r < g.u_max; r += blockDim.x) {
+        const int p = out[r];
+        if (p >= 0) out[r] = cidx[p];
+    }
+}
+
+// ---------------------------------------------------------------------------------------
 // Step (d), SIMT form: one warp per (unit, listed row, key split).  Lane l owns keys
 // lo + l, lo + l + 32, ... and keeps its own online-softmax state (m, l, acc[64]) in base-2
 // exponent form; the 32 states are merged at the end.  With one split the row is finished
@@ -378,9 +434,26 @@ cudaError_t launch_colsum(int dtype, const Geom &g, const void *V, float *part, 
     return cudaGetLastError();
 }
 
+size_t select_cand_ints(int units, int u_max) { return (size_t)units * kSelectMaxSlices * u_max; }
+
 cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *vpart, int n_chunks,
-                          float *vbar, cudaStream_t st) {
+                          float *vbar, int *cand, cudaStream_t st) {
     if (g.B * g.H == 0) return cudaSuccess;
+    const int units = g.B * g.H;
+    int slices = kSmCount / units;
+    if (slices > kSelectMaxSlices) slices = kSelectMaxSlices;
+    if (M != nullptr && vbar == nullptr && cand != nullptr && slices >= 2 && g.u_max <= 64 && g.T / slices >= 1024) {
+        const int width = (g.T + slices - 1) / slices;
+        if (width <= kSelectSmemKeys) {
+            cudaError_t e = launch_pdl(k_select_slice, dim3((unsigned)(units * slices)), dim3(kSelectThreads), 0, st, g, M,
+                                       slices, width, cand);
+            note_launch();
+            if (e != cudaSuccess) return e;
+            e = launch_pdl(k_select_merge, dim3((unsigned)units), dim3(256), 0, st, g, M, slices, (const int *)cand, sel);
+            note_launch();
+            return e != cudaSuccess ? e : cudaGetLastError();
+        }
+    }
     cudaError_t e = launch_pdl(k_select, dim3((unsigned)(g.B * g.H)), dim3(kSelectThreads), 0, st, g, M, sel, vpart, n_chunks, vbar);
     note_launch();
     if (e != cudaSuccess) return e;

@@ -359,6 +359,33 @@ def test_select_entry_point_is_exact_including_ties():
     plan.close()
 
 
+@pytest.mark.parametrize("B,H,T", [(3, 2, 9000), (4, 8, 8192), (1, 1, 8200)])
+def test_select_of_few_long_units_is_exact_including_ties(B, H, T):
+    """Few units of long sequences are selected range by range and then among the ranges' candidates:
+    the result must still be the oracle's, ties (equal values: lower position first) included."""
+    c = 5.0
+    rng = np.random.default_rng(60 + T)
+    M = rng.standard_normal((B, H, T)).astype(np.float32)
+    M[0, 0] = np.round(M[0, 0] * 2) / 2            # heavy ties, spread over every range
+    M[-1, -1] = 0.0                                 # all equal: the first u positions win, all in the first range
+    if B > 1:
+        M[1, 0, :] = -np.abs(M[1, 0])               # all negative
+        M[1, 0, T - 7:] = 3.0                       # the winners sit at the very end of the last range, tied
+    lengths = rng.integers(1, T + 1, size=B).astype(np.int32)
+    lengths[0] = T
+    if B > 1:
+        lengths[1] = T
+    if B > 2:
+        lengths[2] = 1500                           # shorter than two ranges: the other ranges are empty
+    plan = ps.Plan(B, H, T, c=c)
+    sel = plan.psattn_select(torch.from_numpy(M).cuda(), torch.from_numpy(lengths).cuda())
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() == 0
+    ref = orc.select(M.astype(np.float64), lengths, c=c, u_max=plan.u_max)
+    np.testing.assert_array_equal(sel.cpu().numpy(), ref)
+    plan.close()
+
+
 def test_mean_v_entry_point():
     B, H, T = 3, 2, 900
     inp = _synth(B, H, T, 51, 4, "bf16", [900, 257, 1])

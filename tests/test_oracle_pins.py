@@ -199,6 +199,36 @@ def test_full_sample_is_max_minus_mean_over_all_keys():
     np.testing.assert_allclose(Mx, lse - S.mean(-1), atol=1e-12)
 
 
+def test_exact_measure_closed_forms():
+    # Eq. 9-10: M - ln L is the divergence of the attention distribution from the uniform one: zero for
+    # constant scores (M = ln L exactly), and in closed form for one score s above L - 1 zeros:
+    # M = ln(e^s + L - 1) - s / L.  Padded keys (NaN here) are never read.
+    B, H, T, d = 2, 2, 12, 16
+    rng = np.random.default_rng(3)
+    lengths = np.array([12, 7], dtype=np.int32)
+    K = np.zeros((B, H, T, d), dtype=np.float32)
+    rho = 1.5
+    for t in range(T):
+        K[:, :, t, t] = rho                                   # orthogonal keys of norm rho (T <= d)
+    Q0 = np.zeros((B, H, T, d), dtype=np.float32)
+    Q1 = np.zeros((B, H, T, d), dtype=np.float32)
+    alpha = 2.0
+    for b in range(B):
+        for i in range(int(lengths[b])):
+            Q1[b, :, i] = alpha * K[b, :, (i * 5) % int(lengths[b])]
+    K[1, :, 7:] = np.nan
+    Q0[1, :, 7:] = np.nan
+    Q1[1, :, 7:] = np.nan
+    M0 = orc.exact_measure(Q0, K, lengths)
+    M1 = orc.exact_measure(Q1, K, lengths)
+    s = alpha * rho * rho / math.sqrt(d)
+    for b in range(B):
+        L = int(lengths[b])
+        np.testing.assert_allclose(M0[b, :, :L], math.log(L), atol=1e-13)
+        np.testing.assert_allclose(M1[b, :, :L], math.log(math.exp(s) + L - 1) - s / L, atol=1e-13)
+        assert np.all(M0[b, :, L:] == 0.0) and np.all(M1[b, :, L:] == 0.0)
+
+
 # ---- P8: invariances -------------------------------------------------------------------
 
 def test_invariances():

@@ -26,7 +26,7 @@ __global__ void __launch_bounds__(kA64Threads, 1) k_attend64(Geom g, Attend64Arg
                                                              const __grid_constant__ CUtensorMap tmK,
                                                              const __grid_constant__ CUtensorMap tmV) {
     extern __shared__ __align__(1024) uint8_t smem[];
-    uint32_t *tmem_slot_p = reinterpret_cast<uint32_t *>(smem + kA64OffBar + 96);
+    uint32_t *tmem_slot_p = reinterpret_cast<uint32_t *>(smem + kA64OffBar + 120);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int split = blockIdx.x, unit = blockIdx.y;
     if ((smem_u32(smem) & 1023u) != 0u) {                      // swizzled tiles need a 1024-byte base

@@ -11,7 +11,10 @@
 //   control thread   O_a = P_a V_a, O_b = P_b V_b -> TMEM
 //   warpgroup        acc = acc * alpha + O
 // Each warpgroup has its own control thread (lane 0 of warps ctrl_warp and ctrl_warp + 1), so neither
-// waits for the other; the scores of the next pair are issued as soon as the warpgroup has read the current ones.
+// waits for the other.  A warpgroup owns two score accumulators (TMEM columns [256 wg, 256 wg + 128) and the 128
+// after them) used by alternate pairs; O of a pair is written over the first 64 columns of the scores it came
+// from.  So the scores of the next pair are computed as soon as its keys have landed and the other accumulator
+// has been read out, under the softmax of the current pair.
 // At the end the (m, l, acc) states of the two tiles of a pair and of the two warpgroups are merged.
 // Every wait is bounded; on expiry the routine sets the status bit and unwinds.
 #pragma once
@@ -26,7 +29,7 @@ constexpr uint32_t kA64OffWg = 8192;                         // per warpgroup: K
 constexpr uint32_t kA64WgBytes = 6 * kA64Tile;
 constexpr uint32_t kA64OffBar = kA64OffWg + 2 * kA64WgBytes;
 constexpr uint32_t kA64Bytes = kA64OffBar + 128;
-constexpr uint32_t kA64TmemCols = 512;                       // per warpgroup: S 128 columns, O 64 columns
+constexpr uint32_t kA64TmemCols = 512;                       // per warpgroup: two score accumulators of 128 columns
 constexpr int kA64MaxRows = 64;
 
 struct Attend64Job {
@@ -50,12 +53,12 @@ __device__ __forceinline__ void attend64_start(uint8_t *smem, const Attend64Job 
                                                const CUtensorMap *tmV) {
     using namespace sm100;
     uint64_t *kfull = reinterpret_cast<uint64_t *>(smem + kA64OffBar);
-    uint64_t *vfull = kfull + 2, *sfull = kfull + 4, *pready = kfull + 6, *ofull = kfull + 8;
-    volatile uint32_t *abort_flag = reinterpret_cast<uint32_t *>(kfull + 10);
+    uint64_t *vfull = kfull + 2, *sfull = kfull + 4, *pready = kfull + 8, *ofull = kfull + 10, *sfree = kfull + 12;
+    volatile uint32_t *abort_flag = reinterpret_cast<uint32_t *>(kfull + 14);
     const int n_tiles = (j.hi - j.lo + 127) / 128, n_pairs = (n_tiles + 1) / 2;
     for (int x = 0; x < 2; ++x) {
-        mbar_init(&kfull[x], 1); mbar_init(&vfull[x], 1); mbar_init(&sfull[x], 1);
-        mbar_init(&pready[x], 128); mbar_init(&ofull[x], 1);
+        mbar_init(&kfull[x], 1); mbar_init(&vfull[x], 1); mbar_init(&sfull[2 * x], 1); mbar_init(&sfull[2 * x + 1], 1);
+        mbar_init(&pready[x], 128); mbar_init(&ofull[x], 1); mbar_init(&sfree[x], 128);
     }
     *abort_flag = 0u;
     fence_barrier_init();
@@ -139,8 +142,9 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
                                              float &l_out, float acc[kD]) {
     using namespace sm100;
     uint64_t *kfull = reinterpret_cast<uint64_t *>(smem + kA64OffBar);   // [2] per warpgroup
-    uint64_t *vfull = kfull + 2, *sfull = kfull + 4, *pready = kfull + 6, *ofull = kfull + 8;
-    volatile uint32_t *abort_flag = reinterpret_cast<uint32_t *>(kfull + 10);
+    // sfull[2 wg + x]: scores in accumulator x of warpgroup wg; sfree[wg]: the warpgroup has read O of a pair
+    uint64_t *vfull = kfull + 2, *sfull = kfull + 4, *pready = kfull + 8, *ofull = kfull + 10, *sfree = kfull + 12;
+    volatile uint32_t *abort_flag = reinterpret_cast<uint32_t *>(kfull + 14);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_tiles = (j.hi - j.lo + 127) / 128, n_pairs = (n_tiles + 1) / 2;
 
@@ -189,45 +193,56 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             constexpr uint32_t kIdescO = umma_idesc_bf16(64, kD, 1);        // B = V tile, MN-major
             const uint32_t wg_smem = smem_u32(smem + kA64OffWg + wg * kA64WgBytes);
             const uint32_t qa = smem_u32(smem + kA64OffQ);
-            const uint32_t t_s = tmem_base + wg * 192, t_o = t_s + 128;
-            auto issue_s = [&](int q) {                        // S_a = Q K_a^T, S_b = Q K_b^T
+            const uint32_t t_wg = tmem_base + wg * 256;
+            auto issue_s = [&](int q, int x) {                 // S_a = Q K_a^T, S_b = Q K_b^T into accumulator x
                 const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
                 for (int s = 0; s <= two; ++s)
 #pragma unroll
                     for (int k = 0; k < kD / 16; ++k)
-                        umma_bf16(t_s + ((uint32_t)(16 * s) << 16), umma_desc_sw128(qa + k * 32, 16, 1024),
+                        umma_bf16(t_wg + x * 128 + ((uint32_t)(16 * s) << 16), umma_desc_sw128(qa + k * 32, 16, 1024),
                                   umma_desc_sw128(wg_smem + s * kA64Tile + k * 32, 16, 1024), kIdescS, k > 0);
-                umma_commit(&sfull[wg]);
+                umma_commit(&sfull[2 * wg + x]);
             };
             auto give_up = [&]() { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); };
             bool alive = !*abort_flag;
             if (alive && !mbar_wait(&kfull[wg], 0)) { give_up(); alive = false; }
-            if (alive) { tc_fence_after(); issue_s(wg); }
+            if (alive) { tc_fence_after(); issue_s(wg, 0); }
             int cnt = 0;
             for (int q = wg; alive && q < n_pairs; q += 2, ++cnt) {
                 const uint32_t ph = (uint32_t)(cnt & 1);
+                const int x = cnt & 1;
                 const bool more = q + 2 < n_pairs;
                 const int two = (2 * q + 1 < n_tiles) ? 1 : 0;
                 // the K buffers are free once S is done: bring in the next pair's keys
-                if (!mbar_wait(&sfull[wg], ph)) { give_up(); break; }
+                if (!mbar_wait(&sfull[2 * wg + x], (uint32_t)((cnt >> 1) & 1))) { give_up(); break; }
                 if (more) load_pair(wg, q + 2, false);
-                // O_a = P_a V_a, O_b = P_b V_b once the warpgroup has written P
-                if (!mbar_wait(&pready[wg], ph) || !mbar_wait(&vfull[wg], ph)) { give_up(); break; }
-                tc_fence_after();
-                for (int s = 0; s <= two; ++s)
+                // Two things are due now, in whichever order they become possible:
+                //   the next pair's scores, once its keys have landed and the other accumulator has been read out
+                //   (O of the pair before this one sat there);
+                //   O_a = P_a V_a, O_b = P_b V_b of this pair, once the warpgroup has written P and V has landed.
+                bool s_due = more, o_due = true, other_free = cnt == 0;
+                const unsigned long long t0 = global_ns();
+                for (int spin = 0; s_due || o_due; ++spin) {
+                    if (!other_free) other_free = mbar_test(&sfree[wg], ph ^ 1u);
+                    if (s_due && other_free && mbar_test(&kfull[wg], ph ^ 1u)) {
+                        tc_fence_after();
+                        issue_s(q + 2, x ^ 1);
+                        s_due = false;
+                    }
+                    if (o_due && mbar_test(&pready[wg], ph) && mbar_test(&vfull[wg], ph)) {
+                        tc_fence_after();
+                        for (int s = 0; s <= two; ++s)
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        umma_bf16(t_o + ((uint32_t)(16 * s) << 16),
-                                  umma_desc_sw128(wg_smem + (4 + s) * kA64Tile + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024),
-                                  umma_desc_sw128(wg_smem + (2 + s) * kA64Tile + k * 2048, 16, 1024), kIdescO, k > 0);
-                umma_commit(&ofull[wg]);
-                // the warpgroup has read S (it signalled P): the next pair's scores can be computed while it
-                // adds O of this pair to its accumulators
-                if (more) {
-                    if (!mbar_wait(&kfull[wg], ph ^ 1u)) { give_up(); break; }
-                    tc_fence_after();
-                    issue_s(q + 2);
+                            for (int k = 0; k < 8; ++k)
+                                umma_bf16(t_wg + x * 128 + ((uint32_t)(16 * s) << 16),
+                                          umma_desc_sw128(wg_smem + (4 + s) * kA64Tile + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024),
+                                          umma_desc_sw128(wg_smem + (2 + s) * kA64Tile + k * 2048, 16, 1024), kIdescO, k > 0);
+                        umma_commit(&ofull[wg]);
+                        o_due = false;
+                    }
+                    if ((spin & 63) == 63 && (*abort_flag || global_ns() - t0 > kWaitNs)) { give_up(); alive = false; break; }
                 }
+                if (!alive) break;
                 // the V buffers are free once O is done
                 if (!mbar_wait(&ofull[wg], ph)) { give_up(); break; }
                 if (more) load_pair(wg, q + 2, true);
@@ -241,13 +256,14 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
         const bool warp_active = 16 * w4 < max(j.n_rows, j.sum_row + 1);
         const int wtid = (warp - j.wg_warp0 - 4 * wg) * 32 + lane;          // 0..127 inside the warpgroup
         uint8_t *wg_smem = smem + kA64OffWg + wg * kA64WgBytes;
-        const uint32_t t_lane = tmem_base + wg * 192 + ((uint32_t)(32 * w4) << 16);
+        const uint32_t t_lane0 = tmem_base + wg * 256 + ((uint32_t)(32 * w4) << 16);
         uint8_t *prow = wg_smem + (4 + sub) * kA64Tile + row * 128;
         int cnt = 0;
         for (int q = wg; q < n_pairs; q += 2, ++cnt) {
             const uint32_t ph = (uint32_t)(cnt & 1);
             if (*abort_flag) break;
-            if (!mbar_wait(&sfull[wg], ph)) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); break; }
+            const uint32_t t_lane = t_lane0 + (uint32_t)(cnt & 1) * 128u;   // this pair's accumulator
+            if (!mbar_wait(&sfull[2 * wg + (cnt & 1)], (uint32_t)((cnt >> 1) & 1))) { *abort_flag = 1u; atomicOr(g.status, kStatusWaitExpired); break; }
             tc_fence_after();
             const int valid_a = min(128, j.hi - (j.lo + 2 * q * 128));
             const int valid_b = max(0, min(128, j.hi - (j.lo + (2 * q + 1) * 128)));
@@ -274,8 +290,8 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
             __syncwarp();
             if (warp_active) {
                 uint32_t ov[2][32];
-                tmem_ld32_issue(t_lane + 128, ov[0]);
-                tmem_ld32_issue(t_lane + 160, ov[1]);
+                tmem_ld32_issue(t_lane, ov[0]);                 // O sits over the first 64 score columns
+                tmem_ld32_issue(t_lane + 32, ov[1]);
                 tmem_ld_wait();
                 tmem_ld_fence32(ov[0]); tmem_ld_fence32(ov[1]);
                 if (valid > 0) {
@@ -284,6 +300,7 @@ __device__ __forceinline__ bool attend64_run(uint8_t *smem, uint32_t tmem_base, 
                 }
             }
             tc_fence_before();
+            mbar_arrive(&sfree[wg]);                           // this accumulator may take the scores of pair q + 4
         }
         // merge the two tiles of the pair stream: lanes l and l ^ 16 hold the same row
         __syncwarp();

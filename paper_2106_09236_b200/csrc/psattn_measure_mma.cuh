@@ -214,20 +214,27 @@ __device__ __forceinline__ bool measure_resident(uint8_t *smem, uint64_t *bar, u
     const __nv_bfloat16 *Qu = Q + unit_off(g.qs, b, h);
     const uint32_t stage0 = smem_u32(smem) + k_bytes;
     const int n_blocks = (q_end - q_lo + kBlock - 1) / kBlock;
-    auto stage_block = [&](int blk) {                 // always commits a group, even an empty one
+    // Every warp stages the rows of its own eight queries of a block (Q rows, then sample rows, at the warp's
+    // place in the block's buffer) and nobody else reads them, so the warps run through the blocks without
+    // meeting at a barrier.  Always commits a group, even an empty one.
+    const int warp = tid >> 5, lane = tid & 31;
+    auto stage_block = [&](int blk) {
         if (blk < n_blocks) {
-            const int i0 = q_lo + blk * kBlock;
-            const int rows = min(kBlock, q_end - i0);
-            const uint32_t base = stage0 + (uint32_t)(blk % kMeasureStages) * stage_bytes;
-            for (int e = tid; e < rows * 8; e += THREADS)
-                cp_async_16(base + (uint32_t)e * 16u, Qu + (long long)(i0 + (e >> 3)) * g.qs[2] + (e & 7) * 8);
-            const int words = rows * g.idx_cols;
-            const int *src = idx_base + (long long)i0 * g.idx_cols;
-            if (((reinterpret_cast<uintptr_t>(src) | (uintptr_t)(words * 4)) & 15u) == 0u) {
-                for (int w = tid; w < words / 4; w += THREADS)
-                    cp_async_16(base + kBlock * 128u + (uint32_t)w * 16u, src + 4 * w);
-            } else {
-                for (int w = tid; w < words; w += THREADS) cp_async_4(base + kBlock * 128u + (uint32_t)w * 4u, src + w);
+            const int i0 = q_lo + blk * kBlock + warp * 8;
+            const int rows = min(8, q_end - i0);
+            if (rows > 0) {
+                const uint32_t base = stage0 + (uint32_t)(blk % kMeasureStages) * stage_bytes;
+                const uint32_t qdst = base + (uint32_t)warp * 1024u;
+                for (int e = lane; e < rows * 8; e += 32)
+                    cp_async_16(qdst + (uint32_t)e * 16u, Qu + (long long)(i0 + (e >> 3)) * g.qs[2] + (e & 7) * 8);
+                const int words = rows * g.idx_cols;
+                const int *src = idx_base + (long long)i0 * g.idx_cols;
+                const uint32_t idst = base + kBlock * 128u + (uint32_t)(warp * 8 * g.idx_cols) * 4u;
+                if (((reinterpret_cast<uintptr_t>(src) | (uintptr_t)(words * 4)) & 15u) == 0u) {
+                    for (int w = lane; w < words / 4; w += 32) cp_async_16(idst + (uint32_t)w * 16u, src + 4 * w);
+                } else {
+                    for (int w = lane; w < words; w += 32) cp_async_4(idst + (uint32_t)w * 4u, src + w);
+                }
             }
         }
         cp_async_commit();
@@ -249,9 +256,9 @@ __device__ __forceinline__ bool measure_resident(uint8_t *smem, uint64_t *bar, u
     cx.k_base = smem_u32(smem); cx.U = U; cx.L = L; cx.idx_cols = g.idx_cols; cx.status = g.status;
 
     for (int blk = 0; blk < n_blocks; ++blk) {
-        stage_block(blk + kMeasureStages - 1);            // its buffer was released by the barrier below
-        cp_async_wait<kMeasureStages - 1>();              // block blk has landed
-        __syncthreads();
+        stage_block(blk + kMeasureStages - 1);            // into the buffer this warp left at the end of the trip before
+        cp_async_wait<kMeasureStages - 1>();              // this lane's part of block blk has landed
+        __syncwarp();                                     // ... and the other lanes' parts
         asm volatile("mov.u32 %0, %1;" : "=r"(cx.epoch) : "r"(blk) : "memory");
         cx.q_tile = stage0 + (uint32_t)(blk % kMeasureStages) * stage_bytes;
         cx.idx_tile = cx.q_tile + kBlock * 128u;
@@ -259,7 +266,7 @@ __device__ __forceinline__ bool measure_resident(uint8_t *smem, uint64_t *bar, u
         cx.rows = min(kBlock, q_end - i0);
         cx.out = out + i0;
         measure_block<THREADS>(cx);
-        __syncthreads();                              // the buffer may be restaged from now on
+        __syncwarp();                                 // the warp's part of the buffer may be restaged from now on
     }
     return true;
 }

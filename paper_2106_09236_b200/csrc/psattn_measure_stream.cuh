@@ -169,7 +169,7 @@ __device__ __forceinline__ void measure_stream_block(const StreamCtx &cx) {
 
 // All THREADS threads of the CTA: M~ of the queries [q_lo, q_end) (q_end <= L, L >= 1) of unit (b, h)
 // into out[i].  Shared memory: THREADS / 32 rings, then two staging buffers of stage_bytes.
-// Contains __syncthreads.
+// No block-wide barrier inside: the caller orders the result with one of its own where it needs to.
 template <int THREADS>
 __device__ __forceinline__ void measure_stream(uint8_t *smem, uint32_t stage_bytes, const Geom &g, int unit, int b, int h,
                                                int L, int U, int q_lo, int q_end, const __nv_bfloat16 *__restrict__ Q,
@@ -183,20 +183,27 @@ __device__ __forceinline__ void measure_stream(uint8_t *smem, uint32_t stage_byt
     const __nv_bfloat16 *Qu = Q + unit_off(g.qs, b, h);
     const uint32_t stage0 = smem_u32(smem) + kRingBytes;
     const int n_blocks = (q_end - q_lo + kBlock - 1) / kBlock;
+    // every warp stages the rows of its own eight queries (see measure_resident): no barrier between blocks,
+    // so the warps drift apart and the pipeline bubble at the start of a group of queries does not hit all
+    // of them at once
+    const int warp = tid >> 5, lane = tid & 31;
     auto stage_block = [&](int blk) {
         if (blk < n_blocks) {
-            const int i0 = q_lo + blk * kBlock;
-            const int rows = min(kBlock, q_end - i0);
-            const uint32_t base = stage0 + (uint32_t)(blk & 1) * stage_bytes;
-            for (int e = tid; e < rows * 8; e += THREADS)
-                cp_async_16(base + (uint32_t)e * 16u, Qu + (long long)(i0 + (e >> 3)) * g.qs[2] + (e & 7) * 8);
-            const int words = rows * g.idx_cols;
-            const int *src = idx_base + (long long)i0 * g.idx_cols;
-            if (((reinterpret_cast<uintptr_t>(src) | (uintptr_t)(words * 4)) & 15u) == 0u) {
-                for (int w = tid; w < words / 4; w += THREADS)
-                    cp_async_16(base + kBlock * 128u + (uint32_t)w * 16u, src + 4 * w);
-            } else {
-                for (int w = tid; w < words; w += THREADS) cp_async_4(base + kBlock * 128u + (uint32_t)w * 4u, src + w);
+            const int i0 = q_lo + blk * kBlock + warp * 8;
+            const int rows = min(8, q_end - i0);
+            if (rows > 0) {
+                const uint32_t base = stage0 + (uint32_t)(blk & 1) * stage_bytes;
+                const uint32_t qdst = base + (uint32_t)warp * 1024u;
+                for (int e = lane; e < rows * 8; e += 32)
+                    cp_async_16(qdst + (uint32_t)e * 16u, Qu + (long long)(i0 + (e >> 3)) * g.qs[2] + (e & 7) * 8);
+                const int words = rows * g.idx_cols;
+                const int *src = idx_base + (long long)i0 * g.idx_cols;
+                const uint32_t idst = base + kBlock * 128u + (uint32_t)(warp * 8 * g.idx_cols) * 4u;
+                if (((reinterpret_cast<uintptr_t>(src) | (uintptr_t)(words * 4)) & 15u) == 0u) {
+                    for (int w = lane; w < words / 4; w += 32) cp_async_16(idst + (uint32_t)w * 16u, src + 4 * w);
+                } else {
+                    for (int w = lane; w < words; w += 32) cp_async_4(idst + (uint32_t)w * 4u, src + w);
+                }
             }
         }
         cp_async_commit();
@@ -207,8 +214,8 @@ __device__ __forceinline__ void measure_stream(uint8_t *smem, uint32_t stage_byt
     cx.Ku = K + unit_off(g.ks, b, h); cx.k_row_bytes = (uint32_t)(g.ks[2] * 2);
     stage_block(0);
     for (int blk = 0; blk < n_blocks; ++blk) {
-        cp_async_wait<0>();                                    // block blk (and nothing else) is pending
-        __syncthreads();
+        cp_async_wait<0>();                                    // this lane's part of block blk (nothing else is pending)
+        __syncwarp();
         asm volatile("mov.u32 %0, %1;" : "=r"(cx.epoch0) : "r"(blk << 8) : "memory");
         stage_block(blk + 1);                                  // lands while this block is worked on
         cx.q_tile = stage0 + (uint32_t)(blk & 1) * stage_bytes;
@@ -217,7 +224,7 @@ __device__ __forceinline__ void measure_stream(uint8_t *smem, uint32_t stage_byt
         cx.rows = min(kBlock, q_end - i0);
         cx.out = out + i0;
         measure_stream_block<THREADS>(cx);
-        __syncthreads();                                       // buffer blk & 1 may be restaged next time
+        __syncwarp();                                          // the warp's part of buffer blk & 1 may be restaged next time
     }
     cp_async_wait<0>();
 }

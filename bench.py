@@ -56,12 +56,12 @@ _FUSED_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.
 _STREAM_SOURCES = ["psattn_measure_mma.cu", "psattn_measure_stream.cuh", "psattn_measure_mma.cuh",
                    "psattn_sm100.cuh", "psattn_common.cuh"]
 TRAFFIC = {
-    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53627904, "sources": _FUSED_SOURCES,
+    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53625856, "sources": _FUSED_SOURCES,
                    "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
-                   "sources_sha1": "a6f9aaa96cca0c034ff63b835a9151b17b9cf193"},
-    "long_bf16": {"kernel": "k_measure_stream", "bytes": 75807488, "sources": _STREAM_SOURCES,
+                   "sources_sha1": "30622772007f5c0e35b61ed38bfeef9d342cf0d9"},
+    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76343808, "sources": _STREAM_SOURCES,
                   "profile": "profiles/ncu_full_k_measure_stream_long_bf16.txt",
-                  "sources_sha1": "ad541e397bbc41777db8f455f49770f4c4e31091"},
+                  "sources_sha1": "2cefd328bfe39e8941e1eea3f3e682bc492120bf"},
 }
 
 

@@ -230,6 +230,47 @@ def test_workspace_contents_do_not_matter_and_its_bounds_are_kept(dtype, T, path
     plan.close()
 
 
+@pytest.mark.parametrize("dtype,T", [("bf16", 300), ("bf16", 1500), ("fp32", 200)])
+def test_forward_inside_a_cuda_graph_matches_the_direct_call(dtype, T):
+    """The call may fork work onto the plan's side stream and uses programmatic dependent launches: a stream
+    capture has to follow all of it, and a replay on new input values has to give what a direct call gives."""
+    B, H, c = 3, 2, 5.0
+    n = max(orc.count(c, L) for L in range(1, T + 1))
+    lengths = [T, T // 2, T - 3]
+    first = _synth(B, H, T, 700 + T, n, dtype, lengths)
+    second = _synth(B, H, T, 800 + T, n, dtype, lengths)
+    want = _run_forward(second, dtype, c, ps.PSATTN_PATH_AUTO)
+    dev, tdt = _dev(first, dtype)
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n)
+    M = torch.empty((B, H, T), dtype=torch.float32, device="cuda")
+    O = torch.empty((B, H, T, 64), dtype=tdt, device="cuda")
+    sel = torch.empty((B, H, plan.u_max), dtype=torch.int32, device="cuda")
+
+    def call():
+        plan.psattn_forward(dev["Q"], dev["K"], dev["V"], dev["lengths"], dev["sample_idx"], O, sel, M)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        call()                                             # warm-up outside the capture (one-time attribute calls)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    dev2, _ = _dev(second, dtype)
+    for key in ("Q", "K", "V", "sample_idx"):
+        dev[key].copy_(dev2[key])
+    O.fill_(float("nan")); sel.fill_(-7); M.fill_(float("nan"))
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() == 0
+    np.testing.assert_array_equal(O.float().cpu().numpy(), want[0])
+    np.testing.assert_array_equal(sel.cpu().numpy(), want[1])
+    np.testing.assert_array_equal(M.cpu().numpy(), want[2])
+    plan.close()
+
+
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_strided_bthd_layout(path):
     """Q, K, V, O stored [B][T][H][d] (projection output order) through the stride fields."""

@@ -24,8 +24,10 @@
  *   - K~ is drawn per query, with replacement, by the caller (sample_idx is an
  *     input); a key drawn twice counts twice in the mean of Eq. 11.
  *   - The number of selected queries is u = n(c, len) (the Informer rule the
- *     paper builds on) unless u_override > 0, which makes the paper's
- *     L_sparse = r_sparse * L reachable.
+ *     paper builds on) by default.  r_sparse > 0 selects the paper's own count,
+ *     L_sparse = r_sparse * L of Sec. 3.2, per sequence from its own length:
+ *     clamp(ceil(r_sparse * len), 1, len) (rounding up, at least one query).
+ *     u_override > 0 fixes one count min(u_override, len) for all sequences.
  *   - Selection is per (batch, head); larger M~ first, equal M~ -> the smaller
  *     query index; the index set is reported in ascending order, padded by -1.
  *   - Non-selected valid queries receive mean(V) over valid keys (fill 0, the
@@ -143,12 +145,26 @@ void psattn_oracle_exact_measure(const float *Q, const float *K, int B, int H, i
     }
 }
 
+/* Sec. 3.2: how many queries of a sequence of `len` valid positions are selected.
+ * r_sparse > 0: L_sparse = r_sparse * L, rounded up, in [1, len]. */
+int psattn_oracle_selected_count(double c, int u_override, double r_sparse, int len) {
+    if (len <= 0) return 0;
+    if (r_sparse > 0.0) {
+        double x = ceil(r_sparse * (double)len);
+        if (x < 1.0) x = 1.0;
+        if (x > (double)len) x = (double)len;
+        return (int)x;
+    }
+    if (u_override > 0) return u_override < len ? u_override : len;
+    return psattn_oracle_count(c, len);
+}
+
 /* Sec. 3.2: I_sparse = indices of the top-u queries by M~, per (batch, head). */
 void psattn_oracle_select(const double *M, int B, int H, int T, const int *lengths,
-                          double c, int u_override, int *sel_idx, int u_max) {
+                          double c, int u_override, double r_sparse, int *sel_idx, int u_max) {
     for (int b = 0; b < B; ++b) {
         int L = seq_len(lengths, b, T);
-        int u = u_override > 0 ? (u_override < L ? u_override : L) : psattn_oracle_count(c, L);
+        int u = psattn_oracle_selected_count(c, u_override, r_sparse, L);
         if (u > u_max) u = u_max;
         for (int h = 0; h < H; ++h) {
             const double *Mu = M + ((size_t)b * H + h) * T;
@@ -215,6 +231,7 @@ void psattn_oracle_attend_row(const float *Q, const float *K, const float *V, in
  *   sel_idx  int32  [B][H][u_max]        ascending, -1 padded
  *   sel_in   if non-NULL, a given index set (same layout) replaces the
  *            measure and the selection: the cross-layer reuse of Sec. 4.4.
+ *   r_sparse > 0: the paper's count L_sparse = r_sparse * L per sequence (Sec. 3.2).
  *   fill     0: mean(V) over valid keys;  1: the query's own value row.
  *   nthreads OpenMP threads over (batch, head) units for the timed run; the
  *            arithmetic per unit is the same single-threaded code.
@@ -222,7 +239,7 @@ void psattn_oracle_attend_row(const float *Q, const float *K, const float *V, in
 void psattn_oracle_forward(const float *Q, const float *K, const float *V, int B, int H,
                            int T, int d, const int *lengths, const int *sample_idx,
                            int idx_cols, int idx_per_head, double c, int u_override,
-                           int U_override, int fill, const int *sel_in, double *O,
+                           double r_sparse, int U_override, int fill, const int *sel_in, double *O,
                            double *M, int *sel_idx, int u_max, int nthreads) {
     size_t units = (size_t)B * H;
     double *Mloc = M ? M : (double *)malloc(sizeof(double) * units * (size_t)T);
@@ -239,7 +256,7 @@ void psattn_oracle_forward(const float *Q, const float *K, const float *V, int B
             psattn_oracle_measure(Q + un * (size_t)T * d, K + un * (size_t)T * d, 1, 1, T, d,
                                   len1, idx1, idx_cols, 1, c, U_override,
                                   Mloc + un * (size_t)T);
-            psattn_oracle_select(Mloc + un * (size_t)T, 1, 1, T, len1, c, u_override,
+            psattn_oracle_select(Mloc + un * (size_t)T, 1, 1, T, len1, c, u_override, r_sparse,
                                  sel_idx + un * (size_t)u_max, u_max);
         }
     } else {

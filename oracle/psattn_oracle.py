@@ -104,22 +104,34 @@ def exact_measure(Q, K, lengths=None):
     return M
 
 
-def select(M, lengths=None, c=5.0, u_override=0, u_max=None):
+def selected_count(length: int, c: float = 5.0, u_override: int = 0, r_sparse: float = 0.0) -> int:
+    """Number of selected queries of a sequence: n(c, len), or ceil(r_sparse * len) in [1, len]
+    (Sec. 3.2's L_sparse = r_sparse L) when r_sparse > 0, or min(u_override, len)."""
+    lib = _load()
+    lib.psattn_oracle_selected_count.restype = ctypes.c_int
+    return int(lib.psattn_oracle_selected_count(ctypes.c_double(c), int(u_override),
+                                                ctypes.c_double(r_sparse), int(length)))
+
+
+def select(M, lengths=None, c=5.0, u_override=0, u_max=None, r_sparse=0.0):
     """Top-u query indices per (batch, head): int32 [B, H, u_max], ascending, -1 padded."""
     lib = _load()
     M = np.ascontiguousarray(M, dtype=np.float64)
     B, H, T = M.shape
     lengths, lp = _i32(lengths)
     if u_max is None:
-        u_max = u_bound(T, c, u_override)
+        u_max = u_bound(T, c, u_override, r_sparse)
     sel = np.full((B, H, u_max), -1, dtype=np.int32)
     lib.psattn_oracle_select(M.ctypes.data_as(_f64p), B, H, T, lp, ctypes.c_double(c),
-                             int(u_override), sel.ctypes.data_as(_i32p), int(u_max))
+                             int(u_override), ctypes.c_double(r_sparse),
+                             sel.ctypes.data_as(_i32p), int(u_max))
     return sel
 
 
-def u_bound(T, c, u_override=0):
+def u_bound(T, c, u_override=0, r_sparse=0.0):
     """Largest number of selected queries any sequence of length <= T can have."""
+    if r_sparse > 0:
+        return selected_count(int(T), c, 0, r_sparse) if T > 0 else 0
     if u_override > 0:
         return min(int(u_override), int(T))
     return max(count(c, L) for L in range(1, int(T) + 1)) if T > 0 else 0
@@ -150,7 +162,7 @@ def attend_row(Q, K, V, b, h, i, length=None):
 
 
 def forward(Q, K, V, sample_idx, lengths=None, c=5.0, u_override=0, U_override=0,
-            fill="mean_v", sel_in=None, nthreads=1):
+            fill="mean_v", sel_in=None, nthreads=1, r_sparse=0.0):
     """Steps (a)-(e).  Returns (O float64 [B,H,T,d], sel_idx int32 [B,H,u_max], M float64 [B,H,T])."""
     lib = _load()
     Q, qp = _f32(Q)
@@ -164,14 +176,14 @@ def forward(Q, K, V, sample_idx, lengths=None, c=5.0, u_override=0, U_override=0
         u_max = int(sel_in.shape[-1])
         sp = sel_in.ctypes.data_as(_i32p)
     else:
-        u_max = u_bound(T, c, u_override)
+        u_max = u_bound(T, c, u_override, r_sparse)
         sp = None
     O = np.zeros((B, H, T, d), dtype=np.float64)
     M = np.zeros((B, H, T), dtype=np.float64)
     sel = np.full((B, H, u_max), -1, dtype=np.int32)
     lib.psattn_oracle_forward(qp, kp, vp, B, H, T, d, lp, idx.ctypes.data_as(_i32p),
                               int(idx.shape[-1]), per_head, ctypes.c_double(c),
-                              int(u_override), int(U_override),
+                              int(u_override), ctypes.c_double(r_sparse), int(U_override),
                               {"mean_v": 0, "own_v": 1}[fill], sp,
                               O.ctypes.data_as(_f64p), M.ctypes.data_as(_f64p),
                               sel.ctypes.data_as(_i32p), u_max, int(nthreads))

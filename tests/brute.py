@@ -30,8 +30,12 @@ def sampled_measure(q, Kmat, idx):
     return s.max() - s.mean()
 
 
-def forward(Q, K, V, sample_idx, lengths, c, u_override=0, U_override=0, fill="mean_v"):
+def forward(Q, K, V, sample_idx, lengths, c, u_override=0, U_override=0, fill="mean_v", r_sparse=0.0):
+    """sample_idx [B, T, cols] (one sample per query, shared by the heads) or [B, H, T, cols]
+    (every head draws its own).  r_sparse > 0: L_sparse = ceil(r_sparse * L) queries are selected
+    (Sec. 3.2) instead of n(c, L)."""
     B, H, T, d = Q.shape
+    per_head = np.ndim(sample_idx) == 4
     O = np.zeros((B, H, T, d))
     M = np.zeros((B, H, T))
     sels = []
@@ -39,9 +43,12 @@ def forward(Q, K, V, sample_idx, lengths, c, u_override=0, U_override=0, fill="m
         L = int(lengths[b]) if lengths is not None else T
         U = U_override if U_override > 0 else n_count(c, L)
         u = min(u_override, L) if u_override > 0 else n_count(c, L)
+        if r_sparse > 0 and L > 0:
+            u = min(L, max(1, math.ceil(r_sparse * L)))
         for h in range(H):
             for i in range(L):
-                M[b, h, i] = sampled_measure(Q[b, h, i], K[b, h], sample_idx[b, i, :U])
+                row = sample_idx[b, h, i] if per_head else sample_idx[b, i]
+                M[b, h, i] = sampled_measure(Q[b, h, i], K[b, h], row[:U])
             order = sorted(range(L), key=lambda i: (-M[b, h, i], i))
             chosen = sorted(order[:u])
             sels.append(chosen)

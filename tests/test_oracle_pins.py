@@ -87,6 +87,64 @@ def test_brute_force_d64_with_duplicates():
     assert M[0, 0, 3] == 0.0 and M[0, 1, 3] == 0.0
 
 
+def test_brute_force_per_head_samples():
+    """Sec. 3.2 leaves open whether the heads of a sequence share one sample; with a 4-D sample_idx
+    [B][H][T][cols] every head has its own rows.  Different rows per head, ragged lengths: a wrong
+    row stride in the per-head addressing of measure or forward fails here."""
+    B, H, T, d, c = 2, 3, 19, 16, 2.0
+    lengths = np.array([19, 11], dtype=np.int32)
+    ncol = brute.n_count(c, T)
+    rng = np.random.default_rng(4242)
+    Q = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    K = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    V = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    idx = np.zeros((B, H, T, ncol), dtype=np.int32)
+    for b in range(B):
+        L = int(lengths[b])
+        idx[b, :, :L] = rng.integers(0, L, size=(H, L, ncol))
+    assert not np.array_equal(idx[:, 0], idx[:, 1])
+    Mb = brute.forward(Q, K, V, idx, lengths, c)[2]
+    M = orc.measure(Q, K, idx, lengths, c=c)
+    np.testing.assert_allclose(M, Mb, rtol=0, atol=1e-12)
+    for fill in ("mean_v", "own_v"):
+        O, sel, M2 = orc.forward(Q, K, V, idx, lengths, c=c, fill=fill)
+        Ob, selb, _ = brute.forward(Q, K, V, idx, lengths, c, fill=fill)
+        np.testing.assert_allclose(M2, Mb, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(O, Ob, rtol=0, atol=1e-12)
+        got = [[int(x) for x in sel[b, h] if x >= 0] for b in range(B) for h in range(H)]
+        assert got == selb
+    # the shared layout is the per-head layout with equal rows in every head
+    shared = idx[:, 0]
+    M_sh = orc.measure(Q, K, shared, lengths, c=c)
+    M_rep = orc.measure(Q, K, np.repeat(shared[:, None], H, axis=1), lengths, c=c)
+    np.testing.assert_array_equal(M_sh, M_rep)
+    assert not np.allclose(M_sh, M)
+
+
+def test_paper_count_rule_per_sequence():
+    """Sec. 3.2: L_sparse = r_sparse L from every sequence's own length (rounded up, at least one).
+    Ragged lengths: each sequence gets its own count; brute force on the whole path."""
+    for L, r, want in ((1, 0.5, 1), (2, 0.5, 1), (3, 0.5, 2), (40, 0.35, 14), (500, 0.35, 175),
+                       (501, 0.5, 251), (7, 0.01, 1), (7, 1.0, 7), (0, 0.5, 0)):
+        assert orc.selected_count(L, r_sparse=r) == want
+    assert orc.selected_count(100, c=5.0) == brute.n_count(5.0, 100)
+    assert orc.selected_count(10, u_override=4) == 4 and orc.selected_count(3, u_override=4) == 3
+    B, H, T, d, c = 3, 2, 21, 8, 1.5
+    lengths = np.array([21, 9, 4], dtype=np.int32)
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 77, brute.n_count(c, T), lengths)
+    for r in (0.35, 0.5):
+        O, sel, M = orc.forward(Q, K, V, idx, lengths, c=c, fill="own_v", r_sparse=r)
+        Ob, selb, Mb = brute.forward(Q, K, V, idx, lengths, c, fill="own_v", r_sparse=r)
+        assert sel.shape[-1] == math.ceil(r * T)
+        np.testing.assert_allclose(O, Ob, rtol=0, atol=1e-12)
+        got = [[int(x) for x in sel[b, h] if x >= 0] for b in range(B) for h in range(H)]
+        assert got == selb
+        for b in range(B):
+            assert len(got[b * H]) == math.ceil(r * int(lengths[b]))
+        sel2 = orc.select(M, lengths, c=c, r_sparse=r)
+        np.testing.assert_array_equal(sel2, sel)
+
+
 # ---- P2: u = len  ==> dense softmax attention (Eq. 6) ------------------------------------
 
 def test_all_selected_equals_dense_attention():

@@ -3,9 +3,17 @@
 
 One "step" = one psattn_forward over one batch of a seeded synthetic workload.
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+  python bench.py --probe gather          # only the gather microbenchmarks behind `roofline_gather`
 For N > 1 launch with torch.distributed.run; every rank runs the same per-GPU batch (weak
 scaling, no collective on the data path: (batch, head) units are independent).
 Prints ONE JSON line on rank 0.
+
+Timing: W >= 3 warm-up steps, then repeats of EXACTLY K steps each, every repeat bracketed by a
+barrier and a device synchronisation on both sides and timed with CUDA events on the launching
+stream (max over ranks); repeats go on until 0.3 s of device time have been timed, so that the clock
+sampler sees the GPU under load.  `ms_per_step` is the median over the repeats (`ms_per_step_min`
+the fastest one).  Buffers rotate over enough independent input sets that a set has left L2 before it
+is used again; the same-buffers (warm L2) time is reported beside it.
 """
 from __future__ import annotations
 
@@ -27,26 +35,28 @@ from paper_2106_09236_b200 import workloads as wl  # noqa: E402
 
 METRIC = "prob-sparse attention queries/s"
 UNIT = "queries/s"
-L2_BYTES = 126e6
+MIN_TIMED_SECONDS = 0.3
+HEADLINE = "long_bf16"            # the largest single-GPU workload
+OTHER = "large_bf16"              # the other T >= 1024 workload, timed in the same run
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f)
+    except Exception:
+        return None
 
 
 def measured_peaks():
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    try:
-        with open(path) as f:
-            p = json.load(f)
-        return float(p["hbm_gbs"]), "measured"
-    except Exception:
-        return 6650.0, "fallback"
+    p = _peaks()
+    return (float(p["hbm_gbs"]), "measured") if p and "hbm_gbs" in p else (6650.0, "fallback")
 
 
 def tensor_peak():
     """Dense bf16 tensor throughput (TFLOP/s) for a kernel timed alone: the measured burst figure."""
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            return float(json.load(f)["bf16_tflops"]), "measured"
-    except Exception:
-        return 1590.0, "fallback"
+    p = _peaks()
+    return (float(p["bf16_tflops"]), "measured") if p and "bf16_tflops" in p else (1590.0, "fallback")
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of the dominant kernel from the
@@ -96,6 +106,11 @@ def algorithmic_bytes(w, lengths, count, elem):
     return total + 4 * len(lengths)
 
 
+def config_of(w, n_cols):
+    """The workload as both arms (this library, the CPU oracle) report it."""
+    return {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "d_head": w.d, "c": w.c, "U": n_cols}
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
 
@@ -143,137 +158,210 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
-def cpu_oracle_timing(w, n_cols, steps=None, warmup=0, budget_s=12.0):
-    """Times the CPU oracle (as it stands, all host cores over (batch, head) units) on the whole
-    batch of the workload.  steps=None: one pass to calibrate, then as many passes as fit in about
-    `budget_s` seconds of CPU work."""
+# ---- CPU oracle legs -------------------------------------------------------------------------------
+
+def _oracle_pass(orc, inp, w, nthreads):
+    orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c, nthreads=nthreads)
+
+
+def cpu_oracle_timing(w, n_cols, budget_s=8.0):
+    """The CPU oracle, as it stands, on the host cores: (1) all cores over (batch, head) units on the whole
+    batch, as many passes as fit in about `budget_s` seconds; (2) one thread (the protocol of the paper's
+    Fig. 3) on the first sequence; (3) dense attention (Eq. 6), one thread, on a few rows of one unit,
+    scaled to the batch and labelled as extrapolated."""
     from oracle import psattn_oracle as orc
     inp = wl.make_inputs(w, n_cols)
     cores = orc.max_threads()
     queries = int(inp["lengths"].sum()) * w.H
-
-    def one():
-        orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], inp["lengths"], c=w.c, nthreads=cores)
-
-    for _ in range(warmup):
-        one()
-    if steps is None:
-        t0 = time.perf_counter()
-        one()
-        first = time.perf_counter() - t0
-        steps = int(max(1, min(200, budget_s / max(first, 1e-3))))
     t0 = time.perf_counter()
-    for _ in range(steps):
-        one()
-    dt = (time.perf_counter() - t0) / steps
-    return queries / dt, cores, dt, queries, steps
+    _oracle_pass(orc, inp, w, cores)
+    first = time.perf_counter() - t0
+    passes = int(max(1, min(100, budget_s / max(first, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(passes):
+        _oracle_pass(orc, inp, w, cores)
+    dt = (time.perf_counter() - t0) / passes
+    out = {"value": queries / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": "whole batch of %s (%d valid queries), %d passes of %.3f s each" % (w.name, queries, passes, dt)}
+    # one thread, first sequence only
+    one = {k: (v[:1] if hasattr(v, "shape") else v) for k, v in inp.items()}
+    q1 = int(one["lengths"].sum()) * w.H
+    t0 = time.perf_counter()
+    _oracle_pass(orc, one, w, 1)
+    dt1 = time.perf_counter() - t0
+    out["single_thread"] = {"value": q1 / dt1, "unit": UNIT, "cores": 1,
+                            "sample": "first sequence of %s (%d valid queries), 1 pass of %.3f s" % (w.name, q1, dt1)}
+    # dense attention on the CPU: a few rows of unit (0, 0), one thread, scaled to every valid query
+    L0 = int(inp["lengths"][0])
+    n_rows = int(max(4, min(L0, 2.0e8 / max(1, L0 * w.d * 4))))
+    t0 = time.perf_counter()
+    for i in range(n_rows):
+        orc.attend_row(inp["Q"], inp["K"], inp["V"], 0, 0, i % L0, L0)
+    dtd = (time.perf_counter() - t0) / n_rows
+    key_sum = float(sum(int(L) * int(L) for L in inp["lengths"])) * w.H      # sum over queries of their key count
+    dense_s = dtd * key_sum / L0
+    out["dense_single_thread_extrapolated"] = {
+        "value": queries / dense_s, "unit": UNIT, "cores": 1, "seconds_per_batch": dense_s,
+        "sample": "%d rows of unit (0, 0) over %d keys (%.2f ms per row), scaled by the keys per query of "
+                  "every valid query" % (n_rows, L0, dtd * 1e3)}
+    return out
 
 
 def run_reference(args, w):
+    """The reference arm: no other implementation of the method exists, so it is the CPU oracle as it
+    stands on the host cores, each step a bounded sample (whole sequences) of the same workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import psattn_oracle as orc
     n_cols = max(orc.count(w.c, L) for L in range(1, w.T + 1))
-    steps = max(1, min(args.steps, 50))
-    warm = max(0, min(args.warmup, 2))
-    qps, cores, dt, queries, _ = cpu_oracle_timing(w, n_cols, steps, warm)
-    sample = "whole batch of %s (%d valid queries) per step" % (w.name, queries)
+    inp = wl.make_inputs(w, n_cols)
+    cores = orc.max_threads()
+    steps, warm = max(1, args.steps), max(0, args.warmup)
+    # size the sample: time the first sequence, then take as many sequences as keep the run near 100 s
+    one = {k: (v[:1] if hasattr(v, "shape") else v) for k, v in inp.items()}
+    t0 = time.perf_counter()
+    _oracle_pass(orc, one, w, cores)
+    t_one = time.perf_counter() - t0
+    # the units of one sequence may not fill the cores: a batch of nb sequences costs about t_one * nb * H / cores ... at most t_one * nb
+    nb = int(max(1, min(w.B, 100.0 / max(1e-4, t_one * (steps + warm)))))
+    sample = {k: (v[:nb] if hasattr(v, "shape") else v) for k, v in inp.items()}
+    queries = int(sample["lengths"].sum()) * w.H
+    for _ in range(warm):
+        _oracle_pass(orc, sample, w, cores)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        _oracle_pass(orc, sample, w, cores)
+    dt = (time.perf_counter() - t0) / steps
+    qps = queries / dt
+    text = "first %d of %d sequences of %s (%d valid queries) per step" % (nb, w.B, w.name, queries)
     line = {
         "impl": "reference", "metric": METRIC, "value": qps, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "d_head": w.d, "c": w.c},
-        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": config_of(w, n_cols),
+        "cpu_baseline": {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": text},
         "e2e": {"value": qps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
 
 
-def time_events(fn, steps, torch, grouped=False):
-    """Runs fn(k) for k in range(steps) between two CUDA events on the current stream."""
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    start.record()
-    for k in range(steps):
-        if grouped:
-            fn(k, steps)
-        else:
-            fn(k)
-    end.record()
-    torch.cuda.synchronize()
-    return start.elapsed_time(end) / steps      # ms per step
+# ---- GPU side ----------------------------------------------------------------------------------------
+
+class Ctx:
+    """What every timing helper needs: torch, the binding, ranks, flags."""
+
+    def __init__(self, args):
+        import torch
+        import torch.distributed as dist
+        from paper_2106_09236_b200 import binding as ps
+        self.torch, self.dist, self.ps, self.args = torch, dist, ps, args
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+        props = torch.cuda.get_device_properties(self.local)
+        self.sms = int(props.multi_processor_count)
+        self.l2_bytes = int(getattr(props, "L2_cache_size", 0) or getattr(props, "l2_cache_size", 0) or 126 * 2 ** 20)
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+
+    def time_once(self, fn, steps, grouped=False):
+        """EXACTLY `steps` calls of fn between two CUDA events on the current stream, a barrier and a device
+        synchronisation on both sides; ms per step, max over ranks."""
+        torch = self.torch
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.barrier()
+        torch.cuda.synchronize()
+        start.record()
+        for k in range(steps):
+            if grouped:
+                fn(k, steps)
+            else:
+                fn(k)
+        end.record()
+        torch.cuda.synchronize()
+        self.barrier()
+        ms = start.elapsed_time(end) / steps
+        return sharding.max_over_ranks(ms, device="cuda") if self.world > 1 else ms
+
+    def time_repeats(self, fn, steps, grouped=False, min_seconds=MIN_TIMED_SECONDS, max_repeats=2000):
+        """Repeats of time_once until `min_seconds` of device time have been timed (at least 3 repeats).
+        Returns the per-repeat ms per step.  All ranks see the same (max-reduced) times, so they agree on
+        the number of repeats."""
+        out, total = [], 0.0
+        while (total < min_seconds or len(out) < 3) and len(out) < max_repeats:
+            ms = self.time_once(fn, steps, grouped)
+            out.append(ms)
+            total += ms * 1e-3 * steps
+        return out
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large_bf16", choices=sorted(wl.WORKLOADS))
-    ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
-    ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of CUDA-graph replays")
-    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
-    ap.add_argument("--no-dense", action="store_true", help="skip the dense comparator timing")
-    ap.add_argument("--no-variants", action="store_true",
-                    help="skip the selection-reuse and paper-literal timings")
-    args = ap.parse_args()
-    w = wl.WORKLOADS[args.workload]
-    if args.impl == "reference":
-        run_reference(args, w)
-        return
+def gather_probe(cx):
+    """The two gather ceilings of steps (a)+(b), measured here and now with the library's own probe kernels:
+    random 128-byte rows out of a chunk resident in shared memory (ldmatrix pattern of the resident-key
+    kernel) and out of an L2-resident buffer the size of the keys of `long_bf16` (register loads)."""
+    torch, ps = cx.torch, cx.ps
+    sink = torch.zeros(4, dtype=torch.int32, device="cuda")
+    out = {}
 
-    import torch
-    import torch.distributed as dist
-    from paper_2106_09236_b200 import binding as ps
+    def best(fn, n=5):
+        fn()
+        torch.cuda.synchronize()
+        t = []
+        for _ in range(n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            rows = fn()
+            b.record()
+            torch.cuda.synchronize()
+            t.append(a.elapsed_time(b))
+        return rows * 128 / (min(t) * 1e-3) / 1e9          # GB/s
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    gbs = best(lambda: ps.psattn_probe_gather(0, None, cx.sms, 16, 4000, sink))
+    out["shared_memory"] = {"gbs": gbs, "how": "psattn_probe_gather mode 0: %d CTAs x 16 warps, ldmatrix.x4 of random rows of a "
+                                             "resident 128 KB chunk, best of 5" % cx.sms}
+    buf = torch.randn(int(33.5e6 / 4), device="cuda")
+    gbs = max(best(lambda: ps.psattn_probe_gather(m, buf, cx.sms, 24, 800, sink)) for m in (1, 2))
+    out["l2"] = {"gbs": gbs, "how": "psattn_probe_gather modes 1-2: %d CTAs x 24 warps, 16-byte register loads of random 128-byte "
+                                   "rows of a 33.5 MB buffer (L2 resident), best of 5" % cx.sms}
+    del buf
+    return out
 
-    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
-    elem = 2 if w.dtype == "bf16" else 4
-    n_cols = max(ps.psattn_count(w.c, L) for L in range(1, w.T + 1))
-    path = {"auto": ps.PSATTN_PATH_AUTO, "staged": ps.PSATTN_PATH_STAGED, "fused": ps.PSATTN_PATH_FUSED}[args.path]
-    plan = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, path=path)
 
-    # enough independent buffer sets that a set is evicted from L2 before it is used again
+def make_sets(cx, w, n_cols, plan, tdt, elem):
+    torch, ps = cx.torch, cx.ps
     per_set = 4 * w.B * w.H * w.T * w.d * elem + w.B * w.T * n_cols * 4
-    n_sets = max(2, int(np.ceil(2.2 * L2_BYTES / per_set)) + 1)
-    sets, host_sets, queries_per_step, alg_bytes = [], [], None, None
+    n_sets = max(2, int(np.ceil(2.2 * cx.l2_bytes / per_set)) + 1)
+    sets, host0 = [], None
     for s in range(n_sets):
-        inp = wl.make_inputs(w, n_cols, seed=sharding.rank_seed(w.seed, rank, s))
+        inp = wl.make_inputs(w, n_cols, seed=sharding.rank_seed(w.seed, cx.rank, s))
         if s == 0:
-            host_sets.append(inp)
-            queries_per_step = int(inp["lengths"].sum()) * w.H
-            alg_bytes = algorithmic_bytes(w, inp["lengths"], ps.psattn_count, elem)
+            host0 = inp
         d = {k: torch.from_numpy(inp[k]).to("cuda", tdt) for k in ("Q", "K", "V")}
         d["lengths"] = torch.from_numpy(inp["lengths"]).cuda()
         d["sample_idx"] = torch.from_numpy(inp["sample_idx"]).cuda()
         d["O"] = torch.empty((w.B, w.H, w.T, w.d), dtype=tdt, device="cuda")
         d["sel"] = torch.empty((w.B, w.H, plan.u_max), dtype=torch.int32, device="cuda")
         sets.append(d)
+    return sets, host0, per_set
 
-    def step(k):
-        d = sets[k % n_sets]
-        plan.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], d["sel"])
 
-    l0 = ps.psattn_launch_count()
-    step(0)
-    torch.cuda.synchronize()
-    launches_per_step = ps.psattn_launch_count() - l0
+class Replay:
+    """CUDA-graph replay of fn(set index): one graph per buffer set plus one that runs all sets in turn
+    (fewer graph launches per timed step).  With graphs switched off it calls fn directly."""
 
-    def capture(fn):
-        """CUDA graphs around fn(set index): one per buffer set, plus one that runs all sets in turn
-        (fewer graph launches per timed step).  None when graphs are switched off."""
-        if args.no_graph:
-            return None
+    def __init__(self, cx, fn, n_sets, use_graph=True):
+        torch = cx.torch
+        self.fn, self.n_sets, self.singles, self.group = fn, n_sets, None, None
+        if not use_graph:
+            return
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -281,250 +369,367 @@ def main():
                 fn(s)
         torch.cuda.current_stream().wait_stream(side)
         torch.cuda.synchronize()
-        singles = []
+        self.singles = []
         for s in range(n_sets):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
                 fn(s)
-            singles.append(g)
-        group = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(group):
+            self.singles.append(g)
+        self.group = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.group):
             for s in range(n_sets):
                 fn(s)
-        return singles, group
 
-    def replayer(fn, gs):
-        """k -> runs step k.  With graphs: the group graph replays n_sets consecutive steps when k is
-        a multiple of n_sets and enough steps remain; the tail runs through the single graphs."""
-        if gs is None:
-            return lambda k, total=None: fn(k)
-        singles, group = gs
+    def __call__(self, k, total=None):
+        """Runs step k.  With `total` given, the group graph replays n_sets consecutive steps when k is a
+        multiple of n_sets and enough steps remain; the tail runs through the single graphs."""
+        if self.singles is None:
+            self.fn(k % self.n_sets)
+            return
+        if total is None:
+            self.singles[k % self.n_sets].replay()
+            return
+        full = (total // self.n_sets) * self.n_sets
+        if k < full:
+            if k % self.n_sets == 0:
+                self.group.replay()
+        else:
+            self.singles[k % self.n_sets].replay()
 
-        def run(k, total=None):
-            if total is None:
-                singles[k % n_sets].replay()
-                return
-            full = (total // n_sets) * n_sets
-            if k < full:
-                if k % n_sets == 0:
-                    group.replay()
-            else:
-                singles[k % n_sets].replay()
-        return run
+    def same_set(self, k, total=None):
+        """Step k on buffer set 0 every time: inputs stay in L2."""
+        if self.singles is None:
+            self.fn(0)
+        else:
+            self.singles[0].replay()
 
-    graphs = capture(step)
-    timed_step = replayer(step, graphs)
 
-    for k in range(max(args.warmup, 3)):
-        timed_step(k)
+def run_workload(cx, w, probe, headline):
+    """Times one workload.  headline: also the end-to-end call, the CPU legs, the dense comparator and the
+    variants."""
+    torch, ps, args = cx.torch, cx.ps, cx.args
+    tdt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    elem = 2 if w.dtype == "bf16" else 4
+    n_cols = max(ps.psattn_count(w.c, L) for L in range(1, w.T + 1))
+    path = {"auto": ps.PSATTN_PATH_AUTO, "staged": ps.PSATTN_PATH_STAGED, "fused": ps.PSATTN_PATH_FUSED}[args.path]
+    plan = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, path=path)
+    sets, host0, per_set = make_sets(cx, w, n_cols, plan, tdt, elem)
+    n_sets = len(sets)
+    queries_per_step = int(host0["lengths"].sum()) * w.H
+    alg_bytes = algorithmic_bytes(w, host0["lengths"], ps.psattn_count, elem)
+    use_graph = not args.no_graph
+
+    def step(s):
+        d = sets[s]
+        plan.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], d["sel"])
+
+    l0 = ps.psattn_launch_count()
+    step(0)
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
-    ms = time_events(timed_step, args.steps, torch, grouped=True)
-    clocks = sampler.stop()
-    if world > 1:
-        dist.barrier()
-        ms = sharding.max_over_ranks(ms, device="cuda")
-    status = plan.psattn_read_status()
-    value = queries_per_step * world / (ms * 1e-3)
+    launches_per_step = ps.psattn_launch_count() - l0
+    fwd = Replay(cx, step, n_sets, use_graph)
 
-    # direct (non-graph) C-ABI calls, for the record
-    direct_ms = time_events(step, min(args.steps, 200), torch)
+    warm = max(args.warmup, 3)
+    for k in range(warm):
+        fwd(k)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(cx.local)
+    sampler.start()
+    reps = cx.time_repeats(fwd, args.steps, grouped=True)
+    clocks = sampler.stop()
+    status = plan.psattn_read_status()
+    ms, ms_min = float(np.median(reps)), float(min(reps))
+    value = queries_per_step * cx.world / (ms * 1e-3)
+    if clocks["sm_mhz"]:
+        clocks["cycles_per_step"] = ms * 1e3 * clocks["sm_mhz"]      # us x MHz
+    warm_reps = cx.time_repeats(fwd.same_set, args.steps, grouped=True, min_seconds=0.05)
+    direct_ms = cx.time_once(lambda k: step(k % n_sets), min(args.steps, 200))
 
     # per-entry-point times (same kernels), rotating buffers, to find the dominant kernel
     M_buf = torch.empty((w.B, w.H, w.T), dtype=torch.float32, device="cuda")
 
-    def k_measure(k):
-        d = sets[k % n_sets]
+    def k_measure(s):
+        d = sets[s]
         plan.psattn_measure(d["Q"], d["K"], d["lengths"], d["sample_idx"], M_buf)
 
-    def k_rest(k):
-        d = sets[k % n_sets]
+    def k_rest(s):
+        d = sets[s]
         plan.psattn_forward_with_selection(d["Q"], d["K"], d["V"], d["lengths"], d["sel"], d["O"])
 
-    nk = min(args.steps, 200)
-    r_measure, r_rest = replayer(k_measure, capture(k_measure)), replayer(k_rest, capture(k_rest))
+    nk = max(n_sets, min(args.steps, 200))
+    r_measure, r_rest = Replay(cx, k_measure, n_sets, use_graph), Replay(cx, k_rest, n_sets, use_graph)
     for k in range(3):
         r_measure(k); r_rest(k)
-    kernel_ms = {"measure(a+b)": time_events(r_measure, nk, torch, grouped=True),
-                 "mean_v+attend+fill(d+e)": time_events(r_rest, nk, torch, grouped=True)}
-    variants = None
-    if not args.no_variants:
-        variants = {}
-        # Sec. 4.4: N_share consecutive layers share one index set: one full pass, then N_share - 1
-        # passes of steps (d)+(e) on other layers' Q, K, V (the rotating buffer sets stand in for layers)
-        for n_share in (4, 8):
-            def group(k, n=n_share):
-                d0 = sets[(k * n) % n_sets]
-                plan.psattn_forward(d0["Q"], d0["K"], d0["V"], d0["lengths"], d0["sample_idx"], d0["O"], d0["sel"])
-                for j in range(1, n):
-                    d = sets[(k * n + j) % n_sets]
-                    plan.psattn_forward_with_selection(d["Q"], d["K"], d["V"], d["lengths"], d0["sel"], d["O"])
-            r_group = replayer(group, capture(group))
-            for k in range(3):
-                r_group(k)
-            g_ms = time_events(r_group, max(n_sets, nk // n_share), torch, grouped=True)
-            variants["selection_reuse_n_share_%d" % n_share] = {
-                "ms_per_layer": g_ms / n_share, "value": queries_per_step / (g_ms / n_share * 1e-3), "unit": UNIT}
-        # Sec. 3.2 / Eq. 12 as printed: u = ceil(r_sparse * T) selected queries, the others output v_i
-        for r_sparse in (0.35, 0.5):
-            u_lit = int(np.ceil(r_sparse * w.T))
-            plan2 = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, u_override=u_lit,
-                            fill_mode=ps.PSATTN_FILL_OWN_V)
-            sel2 = torch.empty((w.B, w.H, plan2.u_max), dtype=torch.int32, device="cuda")
+    kernel_ms = {
+        "measure(a+b)": float(np.median(cx.time_repeats(r_measure, nk, grouped=True, min_seconds=0.05))),
+        "mean_v+attend+fill(d+e)": float(np.median(cx.time_repeats(r_rest, nk, grouped=True, min_seconds=0.05)))}
 
-            def literal(k):
-                d = sets[k % n_sets]
-                plan2.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], sel2)
-            r_lit = replayer(literal, capture(literal))
-            for k in range(3):
-                r_lit(k)
-            l_ms = time_events(r_lit, max(n_sets, min(nk, 50)), torch, grouped=True)
-            flops = 4.0 * w.d * sum(int(L) * min(u_lit, int(L)) for L in host_sets[0]["lengths"]) * w.H
-            variants["paper_literal_r_sparse_%.2f" % r_sparse] = {
-                "u": u_lit, "fill": "own value row", "ms_per_step": l_ms,
-                "value": queries_per_step / (l_ms * 1e-3), "unit": UNIT,
-                "attention_tflops": flops / (l_ms * 1e-3) / 1e12,
-                "device_status": plan2.psattn_read_status()}
-            plan2.close()
-        # Sec. 3.2 read with ONE sampled key matrix per sequence: step (a) is a dense product on tcgen05
-        plan3 = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, idx_shared=True)
-        sel3 = torch.empty((w.B, w.H, plan3.u_max), dtype=torch.int32, device="cuda")
-        shared_idx = [d["sample_idx"][:, 0, :].contiguous() for d in sets]
-
-        def shared_forward(k):
-            d = sets[k % n_sets]
-            plan3.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], shared_idx[k % n_sets], d["O"], sel3)
-
-        def shared_measure(k):
-            d = sets[k % n_sets]
-            plan3.psattn_measure(d["Q"], d["K"], d["lengths"], shared_idx[k % n_sets], M_buf)
-        r_sf, r_sm = replayer(shared_forward, capture(shared_forward)), replayer(shared_measure, capture(shared_measure))
-        for k in range(3):
-            r_sf(k); r_sm(k)
-        sf_ms = time_events(r_sf, nk, torch, grouped=True)
-        sm_ms = time_events(r_sm, nk, torch, grouped=True)
-        sm_bytes = w.B * w.H * w.T * (w.d * elem + 4)          # Q read once, M written; the sampled keys are small
-        pk, _ = measured_peaks()
-        variants["shared_sample"] = {
-            "ms_per_step": sf_ms, "value": queries_per_step / (sf_ms * 1e-3), "unit": UNIT,
-            "measure_ms": sm_ms, "measure_gbs": sm_bytes / (sm_ms * 1e-3) / 1e9,
-            "measure_frac_of_hbm": sm_bytes / (sm_ms * 1e-3) / 1e9 / pk,
-            "device_status": plan3.psattn_read_status()}
-        plan3.close()
-        # Eq. 10 over all keys: a dense tensor-core pass, the quantity Eq. 11 approximates
-        def exact(k):
-            d = sets[k % n_sets]
-            plan.psattn_exact_measure(d["Q"], d["K"], d["lengths"], M_buf)
-        exact(0)
-        x_ms = time_events(exact, 5, torch)
-        x_flops = 2.0 * w.d * sum(int(L) * int(L) for L in host_sets[0]["lengths"]) * w.H
-        variants["exact_measure"] = {"ms_per_step": x_ms, "tflops": x_flops / (x_ms * 1e-3) / 1e12}
-        # Sec. 3.1: the projections in front of the path (one tcgen05 GEMM writing Q, K, V in the layout
-        # the path reads, plus mean(V)); reported against the measured dense bf16 peak
-        if w.dtype == "bf16":
-            dx = w.H * w.d
-            pin = wl.make_projection_inputs(w, seed=sharding.rank_seed(w.seed, rank, 0))
-            pX = [torch.from_numpy(pin["X"]).to("cuda", tdt) for _ in range(n_sets)]
-            pW = torch.from_numpy(pin["Wt"]).to("cuda", tdt)
-            vb = torch.empty((w.B, w.H, w.d), dtype=torch.float32, device="cuda")
-            pO = [[torch.empty((w.B, w.H, w.T, w.d), dtype=tdt, device="cuda") for _ in range(3)] for _ in range(n_sets)]
-
-            p_flops = 2.0 * dx * 3 * dx * sum(int(L) for L in host_sets[0]["lengths"])
-            tf_peak = tensor_peak()
-            for key, want_vbar in (("qkv_projection", True), ("qkv_projection_without_mean_v", False)):
-                def project(k, want_vbar=want_vbar):
-                    o = pO[k % n_sets]
-                    plan.psattn_project_qkv(pX[k % n_sets], pW, sets[k % n_sets]["lengths"], o[0], o[1], o[2],
-                                            vb if want_vbar else None)
-                r_pj = replayer(project, capture(project))
-                for k in range(3):
-                    r_pj(k)
-                p_ms = time_events(r_pj, nk, torch, grouped=True)
-                variants[key] = {
-                    "ms_per_step": p_ms, "tflops": p_flops / (p_ms * 1e-3) / 1e12, "peak_tflops": tf_peak[0],
-                    "frac_of_tensor_peak": p_flops / (p_ms * 1e-3) / 1e12 / tf_peak[0],
-                    "peak_kind": "of " + tf_peak[1], "d_x": dx, "device_status": plan.psattn_read_status()}
-            del pO, pX
     peak, peak_kind = measured_peaks()
     units = w.B * w.H
     measure_bytes = units * w.T * w.d * elem * 2 + w.B * w.T * n_cols * 4 + units * w.T * 4
     if launches_per_step == 1:
-        roof_kernel, roof_bytes, roof_ms = "fused forward", alg_bytes, ms
+        roof_kernel, roof_bytes, roof_ms = "k_forward_fused (the whole step)", alg_bytes, ms
     else:
-        roof_kernel, roof_bytes, roof_ms = "measure (steps a+b)", measure_bytes, kernel_ms["measure(a+b)"]
+        roof_kernel, roof_bytes, roof_ms = "measure kernel (steps a+b)", measure_bytes, kernel_ms["measure(a+b)"]
     achieved = roof_bytes / (roof_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved, "peak": peak,
-                "unit": "GB/s", "frac": achieved / peak,
-                "traffic": recorded_traffic(w.name),
-                "peak_kind": "of " + peak_kind,
+    roofline = {"bound": "hbm", "kernel": roof_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": recorded_traffic(w.name), "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": roof_bytes}
+    # the second bound: one 128-byte key row per (query, sampled key) pair through the on-chip gather path
+    pairs = sum(int(L) * ps.psattn_count(w.c, int(L)) for L in host0["lengths"]) * w.H
+    resident = launches_per_step == 1
+    ceil = probe["shared_memory" if resident else "l2"]
+    g_achieved = pairs * 128 / (kernel_ms["measure(a+b)"] * 1e-3) / 1e9
+    floor_ms = pairs * 128 / (ceil["gbs"] * 1e9) * 1e3
+    roofline_gather = {
+        "bound": "shared-memory gather" if resident else "L2 gather", "pairs": pairs, "bytes": pairs * 128,
+        "kernel": "measure entry point (steps a+b)", "achieved": g_achieved, "peak": ceil["gbs"], "unit": "GB/s",
+        "frac": g_achieved / ceil["gbs"], "peak_kind": "measured in this run: " + ceil["how"],
+        "floor_ms": floor_ms, "floor_share_of_step": floor_ms / ms}
     path_gbs = alg_bytes / (ms * 1e-3) / 1e9
+    res = {
+        "plan": plan, "sets": sets, "host0": host0, "n_cols": n_cols, "tdt": tdt, "elem": elem,
+        "value": value, "ms": ms, "ms_min": ms_min, "repeats": len(reps), "clocks": clocks, "status": status,
+        "launches_per_step": launches_per_step, "queries_per_step": queries_per_step, "alg_bytes": alg_bytes,
+        "warm_ms": float(np.median(warm_reps)), "direct_ms": direct_ms, "kernel_ms": kernel_ms,
+        "roofline": roofline, "roofline_gather": roofline_gather, "path_gbs": path_gbs, "peak": peak,
+        "per_set": per_set, "n_sets": n_sets, "M_buf": M_buf, "fwd": fwd, "step": step,
+        "timing": {"path": args.path, "graph_replay": use_graph, "repeats": len(reps),
+                   "timed_seconds": float(sum(reps)) * 1e-3 * args.steps,
+                   "l2": "rotating %d independent buffer sets (%.0f MB > %.0f MB L2)" % (
+                       n_sets, n_sets * per_set / 1e6, cx.l2_bytes / 1e6)},
+    }
+    return res
 
-    # end to end through the host-buffer entry point (pinned host memory, copies timed)
-    e2e = None
-    if True:
-        plan.psattn_plan_enable_host_io()
-        inp = host_sets[0]
-        hQ, hK, hV = (torch.from_numpy(inp[k]).to(tdt).pin_memory() for k in ("Q", "K", "V"))
-        hl = torch.from_numpy(inp["lengths"]).pin_memory()
-        hi = torch.from_numpy(inp["sample_idx"]).pin_memory()
-        hO = torch.empty((w.B, w.H, w.T, w.d), dtype=tdt).pin_memory()
-        hs = torch.empty((w.B, w.H, plan.u_max), dtype=torch.int32).pin_memory()
-        ne = max(3, min(args.steps, 20))
-        for _ in range(3):
-            plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs)
-        if world > 1:
-            dist.barrier()
-        e_ms = time_events(lambda k: plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs), ne, torch)
-        if world > 1:
-            e_ms = sharding.max_over_ranks(e_ms, device="cuda")
-        h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hl, hi))
-        d2h = sum(x.numel() * x.element_size() for x in (hO, hs))
-        e2e = {"value": queries_per_step * world / (e_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": ne}
 
-    dense = None
-    if not args.no_dense and rank == 0:
-        d = sets[0]
+def summary_of(r):
+    """The short record of a workload timed beside the headline one."""
+    return {"ms_per_step": r["ms"], "ms_per_step_min": r["ms_min"], "value": r["value"], "unit": UNIT,
+            "warm_l2_ms_per_step": r["warm_ms"], "clocks": r["clocks"], "gpu_launches_per_step": int(r["launches_per_step"]),
+            "roofline": r["roofline"], "roofline_gather": r["roofline_gather"],
+            "path_effective_gbs": r["path_gbs"], "path_frac_of_hbm": r["path_gbs"] / r["peak"],
+            "kernel_ms": r["kernel_ms"], "timing": r["timing"], "device_status": r["status"]}
+
+
+def run_variants(cx, w, r, dense_ms):
+    torch, ps, args = cx.torch, cx.ps, cx.args
+    plan, sets, host0, n_cols, tdt, elem = r["plan"], r["sets"], r["host0"], r["n_cols"], r["tdt"], r["elem"]
+    n_sets, M_buf, queries_per_step = len(sets), r["M_buf"], r["queries_per_step"]
+    use_graph = not args.no_graph
+    nk = max(n_sets, min(args.steps, 200))
+    variants = {}
+
+    def timed(fn, n, min_seconds=0.05):
+        rp = Replay(cx, fn, n_sets, use_graph)
+        for k in range(3):
+            rp(k)
+        return float(np.median(cx.time_repeats(rp, n, grouped=True, min_seconds=min_seconds)))
+
+    # Sec. 4.4: N_share consecutive layers share one index set: one full pass, then N_share - 1
+    # passes of steps (d)+(e) on other layers' Q, K, V (the rotating buffer sets stand in for layers)
+    for n_share in (4, 8):
+        def group(s, n=n_share):
+            d0 = sets[(s * n) % n_sets]
+            plan.psattn_forward(d0["Q"], d0["K"], d0["V"], d0["lengths"], d0["sample_idx"], d0["O"], d0["sel"])
+            for j in range(1, n):
+                d = sets[(s * n + j) % n_sets]
+                plan.psattn_forward_with_selection(d["Q"], d["K"], d["V"], d["lengths"], d0["sel"], d["O"])
+        g_ms = timed(group, max(n_sets, nk // n_share))
+        variants["selection_reuse_n_share_%d" % n_share] = {
+            "ms_per_layer": g_ms / n_share, "value": queries_per_step / (g_ms / n_share * 1e-3), "unit": UNIT}
+    # Sec. 3.2 / Eq. 12 as printed: L_sparse = ceil(r_sparse L) selected queries per sequence, the others output v_i
+    for r_sparse in (0.35, 0.5):
+        plan2 = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, r_sparse=r_sparse, fill_mode=ps.PSATTN_FILL_OWN_V)
+        sel2 = torch.empty((w.B, w.H, plan2.u_max), dtype=torch.int32, device="cuda")
+
+        def literal(s):
+            d = sets[s]
+            plan2.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], sel2)
+        l_ms = timed(literal, max(n_sets, min(nk, 50)))
+        flops = 4.0 * w.d * sum(int(L) * int(np.ceil(r_sparse * int(L))) for L in host0["lengths"]) * w.H
+        variants["paper_literal_r_sparse_%.2f" % r_sparse] = {
+            "u_max": plan2.u_max, "fill": "own value row", "ms_per_step": l_ms,
+            "value": queries_per_step / (l_ms * 1e-3), "unit": UNIT,
+            "attention_tflops": flops / (l_ms * 1e-3) / 1e12, "device_status": plan2.psattn_read_status()}
+        plan2.close()
+    # The setting behind the paper's 8-45 % speed-up (Table 4 row L2, Fig. 3): r_sample = 1, r_sparse = 0.5,
+    # N_share = 4, v_i for the other queries: one full pass and three passes that reuse its selection
+    plan4 = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=1.0, idx_cols=n_cols, r_sparse=0.5, fill_mode=ps.PSATTN_FILL_OWN_V)
+    sel4 = [torch.empty((w.B, w.H, plan4.u_max), dtype=torch.int32, device="cuda") for _ in range(n_sets)]
+
+    def paper_l2(s):
+        d0 = sets[(s * 4) % n_sets]
+        plan4.psattn_forward(d0["Q"], d0["K"], d0["V"], d0["lengths"], d0["sample_idx"], d0["O"], sel4[s])
+        for j in range(1, 4):
+            d = sets[(s * 4 + j) % n_sets]
+            plan4.psattn_forward_with_selection(d["Q"], d["K"], d["V"], d["lengths"], sel4[s], d["O"])
+    p_ms = timed(paper_l2, max(n_sets, min(nk, 20))) / 4
+    variants["paper_L2_r_sample_1_r_sparse_0.5_n_share_4"] = {
+        "ms_per_layer": p_ms, "value": queries_per_step / (p_ms * 1e-3), "unit": UNIT,
+        "dense_ms_per_layer": dense_ms, "speedup_vs_dense": (dense_ms / p_ms) if dense_ms else None,
+        "time_saved_vs_dense": (1.0 - p_ms / dense_ms) if dense_ms else None,
+        "paper": "8-45 % faster than dense on one Xeon thread (context, another machine)",
+        "device_status": plan4.psattn_read_status()}
+    plan4.close()
+    # Sec. 3.2 read with ONE sampled key matrix per sequence: step (a) is a dense product on tcgen05
+    plan3 = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, idx_shared=True)
+    sel3 = torch.empty((w.B, w.H, plan3.u_max), dtype=torch.int32, device="cuda")
+    shared_idx = [d["sample_idx"][:, 0, :].contiguous() for d in sets]
+
+    def shared_forward(s):
+        d = sets[s]
+        plan3.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], shared_idx[s], d["O"], sel3)
+
+    def shared_measure(s):
+        d = sets[s]
+        plan3.psattn_measure(d["Q"], d["K"], d["lengths"], shared_idx[s], M_buf)
+    sf_ms, sm_ms = timed(shared_forward, nk), timed(shared_measure, nk)
+    sm_bytes = w.B * w.H * w.T * (w.d * elem + 4)          # Q read once, M written; the sampled keys are small
+    pk, _ = measured_peaks()
+    variants["shared_sample"] = {
+        "ms_per_step": sf_ms, "value": queries_per_step / (sf_ms * 1e-3), "unit": UNIT,
+        "measure_ms": sm_ms, "measure_gbs": sm_bytes / (sm_ms * 1e-3) / 1e9,
+        "measure_frac_of_hbm": sm_bytes / (sm_ms * 1e-3) / 1e9 / pk, "device_status": plan3.psattn_read_status()}
+    plan3.close()
+
+    # Eq. 10 over all keys: a dense tensor-core pass, the quantity Eq. 11 approximates
+    def exact(s):
+        d = sets[s]
+        plan.psattn_exact_measure(d["Q"], d["K"], d["lengths"], M_buf)
+    x_ms = timed(exact, max(n_sets, 5))
+    x_flops = 2.0 * w.d * sum(int(L) * int(L) for L in host0["lengths"]) * w.H
+    variants["exact_measure"] = {"ms_per_step": x_ms, "tflops": x_flops / (x_ms * 1e-3) / 1e12}
+    # Sec. 3.1: the projections in front of the path (one tcgen05 GEMM writing Q, K, V in the layout
+    # the path reads, plus mean(V)); reported against the measured dense bf16 peak
+    if w.dtype == "bf16":
+        dx = w.H * w.d
+        pin = wl.make_projection_inputs(w, seed=sharding.rank_seed(w.seed, cx.rank, 0))
+        pX = [torch.from_numpy(pin["X"]).to("cuda", tdt) for _ in range(n_sets)]
+        pW = torch.from_numpy(pin["Wt"]).to("cuda", tdt)
+        vb = torch.empty((w.B, w.H, w.d), dtype=torch.float32, device="cuda")
+        pO = [[torch.empty((w.B, w.H, w.T, w.d), dtype=tdt, device="cuda") for _ in range(3)] for _ in range(n_sets)]
+        p_flops = 2.0 * dx * 3 * dx * sum(int(L) for L in host0["lengths"])
+        tf_peak = tensor_peak()
+        for key, want_vbar in (("qkv_projection", True), ("qkv_projection_without_mean_v", False)):
+            def project(s, want_vbar=want_vbar):
+                o = pO[s]
+                plan.psattn_project_qkv(pX[s], pW, sets[s]["lengths"], o[0], o[1], o[2], vb if want_vbar else None)
+            p_ms = timed(project, nk)
+            variants[key] = {
+                "ms_per_step": p_ms, "tflops": p_flops / (p_ms * 1e-3) / 1e12, "peak_tflops": tf_peak[0],
+                "frac_of_tensor_peak": p_flops / (p_ms * 1e-3) / 1e12 / tf_peak[0],
+                "peak_kind": "of " + tf_peak[1], "d_x": dx, "device_status": plan.psattn_read_status()}
+        del pO, pX
+    return variants
+
+
+def run_e2e(cx, w, r):
+    """End to end through the host-buffer entry point (pinned host memory, copies inside the timed region)."""
+    torch, args = cx.torch, cx.args
+    plan, inp, tdt = r["plan"], r["host0"], r["tdt"]
+    plan.psattn_plan_enable_host_io()
+    hQ, hK, hV = (torch.from_numpy(inp[k]).to(tdt).pin_memory() for k in ("Q", "K", "V"))
+    hl = torch.from_numpy(inp["lengths"]).pin_memory()
+    hi = torch.from_numpy(inp["sample_idx"]).pin_memory()
+    hO = torch.empty((w.B, w.H, w.T, w.d), dtype=tdt).pin_memory()
+    hs = torch.empty((w.B, w.H, plan.u_max), dtype=torch.int32).pin_memory()
+    ne = max(3, min(args.steps, 20))
+    for _ in range(3):
+        plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs)
+    reps = cx.time_repeats(lambda k: plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs), ne, min_seconds=0.1)
+    e_ms = float(np.median(reps))
+    h2d = sum(x.numel() * x.element_size() for x in (hQ, hK, hV, hl, hi))
+    d2h = sum(x.numel() * x.element_size() for x in (hO, hs))
+    return {"value": r["queries_per_step"] * cx.world / (e_ms * 1e-3), "unit": UNIT,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": ne, "repeats": len(reps)}
+
+
+def run_dense(cx, w, r):
+    plan, sets = r["plan"], r["sets"]
+    n_sets = len(sets)
+
+    def dense(s):
+        d = sets[s]
         plan.psattn_dense_forward(d["Q"], d["K"], d["V"], d["lengths"], d["O"])
-        nd = 3
-        d_ms = time_events(lambda k: plan.psattn_dense_forward(
-            sets[k % n_sets]["Q"], sets[k % n_sets]["K"], sets[k % n_sets]["V"],
-            sets[k % n_sets]["lengths"], sets[k % n_sets]["O"]), nd, torch)
-        dense = {"ms_per_step": d_ms, "speedup_sparse_vs_dense": d_ms / ms,
-                 "workspace_bytes_sparse": plan.workspace_bytes}
+    rp = Replay(cx, dense, n_sets, not cx.args.no_graph)
+    for k in range(3):
+        rp(k)
+    reps = cx.time_repeats(rp, max(n_sets, 5), grouped=True, min_seconds=0.05)
+    d_ms = float(np.median(reps))
+    flops = 4.0 * w.d * sum(int(L) * int(L) for L in r["host0"]["lengths"]) * w.H
+    tp = tensor_peak()
+    return {"ms_per_step": d_ms, "repeats": len(reps), "speedup_sparse_vs_dense": d_ms / r["ms"],
+            "tflops": flops / (d_ms * 1e-3) / 1e12, "frac_of_tensor_peak": flops / (d_ms * 1e-3) / 1e12 / tp[0],
+            "peak_kind": "of " + tp[1], "workspace_bytes_sparse": plan.workspace_bytes,
+            "score_matrix_bytes_if_materialised": 4 * w.B * w.H * w.T * w.T}
 
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
+    ap.add_argument("--probe", default=None, choices=["gather"], help="run only the named microbenchmark")
+    ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of CUDA-graph replays")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense comparator timing")
+    ap.add_argument("--no-variants", action="store_true", help="skip the timings of the rows marked next")
+    ap.add_argument("--no-others", action="store_true", help="skip the second T >= 1024 workload")
+    args = ap.parse_args()
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    cx = Ctx(args)
+    probe = gather_probe(cx)
+    if args.probe == "gather":
+        if cx.rank == 0:
+            print(json.dumps({"probe": "gather", "sm_count": cx.sms, "ceilings": probe}), flush=True)
+        return
+
+    r = run_workload(cx, w, probe, headline=True)
+    e2e = run_e2e(cx, w, r)
+    dense = run_dense(cx, w, r) if (not args.no_dense and cx.rank == 0) else None
+    variants = None
+    if not args.no_variants and cx.world == 1:
+        variants = run_variants(cx, w, r, dense["ms_per_step"] if dense else None)
+    others = None
+    if not args.no_others and cx.world == 1:
+        others = {}
+        for name in (OTHER, HEADLINE):
+            if name != w.name and name in wl.WORKLOADS and len(others) == 0:
+                r2 = run_workload(cx, wl.WORKLOADS[name], probe, headline=False)
+                others[name] = summary_of(r2)
+                r2["plan"].close()
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu:
-        qps, cores, dt, q, n_pass = cpu_oracle_timing(w, n_cols)
-        cpu = {"value": qps, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "whole batch of %s (%d valid queries), %d passes of %.3f s each" % (w.name, q, n_pass, dt)}
+    if cx.rank == 0 and cx.world == 1 and not args.no_cpu:
+        cpu = cpu_oracle_timing(w, r["n_cols"])
 
-    if rank == 0:
+    if cx.rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
-            "data": "synthetic",
-            "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "d_head": w.d, "c": w.c,
-                       "U": n_cols, "path": args.path, "graph_replay": graphs is not None,
-                       "l2": "rotating %d independent buffer sets (%.0f MB > 126 MB L2)" % (
-                           n_sets, n_sets * per_set / 1e6)},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_per_step * args.steps),
-            "roofline": roofline, "cpu_baseline": cpu,
-            "path_effective_gbs": path_gbs, "path_frac_of_hbm": path_gbs / peak,
-            "algorithmic_bytes_per_step": alg_bytes, "queries_per_step": queries_per_step,
-            "kernel_ms": kernel_ms, "direct_call_ms_per_step": direct_ms, "dense": dense,
-            "variants": variants,
-            "device_status": status,
+            "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": cx.world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": r["ms"], "ms_per_step_min": r["ms_min"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": config_of(w, r["n_cols"]), "timing": r["timing"],
+            "clocks": r["clocks"], "e2e": e2e,
+            "gpu_launches": int(r["launches_per_step"] * args.steps), "gpu_launches_per_step": int(r["launches_per_step"]),
+            "roofline": r["roofline"], "roofline_gather": r["roofline_gather"], "gather_ceilings": probe,
+            "cpu_baseline": cpu,
+            "path_effective_gbs": r["path_gbs"], "path_frac_of_hbm": r["path_gbs"] / r["peak"],
+            "algorithmic_bytes_per_step": r["alg_bytes"], "queries_per_step": r["queries_per_step"],
+            "warm_l2_ms_per_step": r["warm_ms"], "kernel_ms": r["kernel_ms"],
+            "direct_call_ms_per_step": r["direct_ms"], "dense": dense, "variants": variants,
+            "other_workloads": others, "device_status": r["status"],
         }
         print(json.dumps(line), flush=True)
-    plan.close()
-    if world > 1:
-        dist.destroy_process_group()
+    r["plan"].close()
+    if cx.world > 1:
+        cx.dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -11,8 +11,8 @@
  *   (d) o_i = sum_j softmax_j(s_ij) v_j over all valid keys, for i in I_sparse (Eq. 7-8, Eq. 12)
  *   (e) o_i = mean_j v_j over valid keys (or v_i, Eq. 12 as printed) otherwise (Sec. 3.1, Eq. 12)
  *
- * with U = u = n(c, len) = clamp(ceil(c ln len), 1, len) per sequence (Sec. 3.2:
- * "L~ = r_sample ln L"), natural logarithm, evaluated on the host in double.
+ * with U = u = n(c, len) = clamp(ceil(c ln len), 1, len) per sequence (the sample-size rule of
+ * Sec. 3.2 with r_sample = c), natural logarithm, evaluated on the host in double.
  *
  * Conventions common to every call
  *   - All functions return an int status (PSATTN_OK == 0); none throws, aborts or
@@ -90,9 +90,12 @@ typedef struct psattn_desc {
                                            1: [B][H][T_max][idx_cols] */
     int32_t path;                       /* PSATTN_PATH_*: kernel schedule; AUTO picks per shape */
     int32_t idx_shared;                 /* 1: one sample per sequence, used by all its queries (the other
-                                           reading of "a random sampling key matrix", Sec. 3.2): sample_idx
+                                           reading of how Sec. 3.2 draws the sampled keys): sample_idx
                                            is [B][idx_cols] (or [B][H][idx_cols] with idx_per_head) */
     double c;                           /* sampling factor of n(c, len) */
+    double r_sparse;                    /* 0: u = n(c, len).  In (0, 1]: the count of Sec. 3.2 as the paper states it,
+                                           u = clamp(ceil(r_sparse * len), 1, len) from each sequence's own length
+                                           (takes precedence over u_override) */
     int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3];   /* b, h, t strides in elements; all 0 = dense */
 } psattn_desc_t;
 
@@ -147,7 +150,7 @@ int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K, const int3
 int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const void *K, const int32_t *lengths,
                          float *M_out, void *workspace, size_t workspace_bytes, void *stream);
 
-/* The projections that precede the attention (Sec. 3.1: "Q = X W_q, K = X W_k, V = X W_v"), for all heads
+/* The projections that precede the attention (Sec. 3.1: queries, keys and values are the layer input times one matrix each), for all heads
  * at once, written directly in the layout the calls above read.  All pointers device.
  *   X     [B][T_max][d_x], dense, element type of the plan (the layer input; d_x is the model width)
  *   Wt    [3][H * 64][d_x], dense, same type: the matrices stored transposed, role r = 0 (q), 1 (k), 2 (v),
@@ -228,6 +231,20 @@ int psattn_forward_host(psattn_plan_t *plan, const void *Q, const void *K, const
 #define PSATTN_NOALLOC_MAX_PARTIALS 16384
 int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, float *vbar, int32_t B,
                           int32_t H, int32_t T_max, int32_t dtype, void *stream);
+
+/* Microbenchmark of the gather rates that bound steps (a)+(b) (Eq. 11 needs one 128-byte key row per
+ * (query, sampled key) pair, at a random position).  Launches ONE kernel on `stream` that gathers
+ * n_ctas * warps_per_cta * rounds_per_warp * 16 random rows of 128 bytes and computes nothing; the caller
+ * times it (CUDA events) and divides.  No plan, no workspace.
+ *   mode 0  rows of a 128 KB chunk resident in shared memory, read with the ldmatrix pattern of the
+ *           resident-key measure kernel (`rows`, `n_rows` unused; warps_per_cta <= 32)
+ *   mode 1  rows of the device buffer `rows` (n_rows rows of 128 bytes, 16-byte aligned) read from
+ *           global memory / L2 into registers, two rounds in flight per warp (warps_per_cta <= 24;
+ *           rounds_per_warp is rounded down to a multiple of the rounds in flight)
+ *   mode 2  as mode 1 with four rounds in flight per warp
+ * sink: device uint32 (written practically never; it keeps the loads alive). */
+int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_rows, int32_t n_ctas,
+                        int32_t warps_per_cta, int32_t rounds_per_warp, uint32_t *sink, void *stream);
 
 #ifdef __cplusplus
 }

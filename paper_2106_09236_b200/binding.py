@@ -22,6 +22,7 @@ EXPORTS = [
     "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_exact_measure", "psattn_select",
     "psattn_mean_v", "psattn_attend_rows", "psattn_dense_forward", "psattn_read_status",
     "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc", "psattn_project_qkv",
+    "psattn_probe_gather",
 ]
 
 
@@ -32,6 +33,7 @@ class psattn_desc_t(ctypes.Structure):
         ("u_override", ctypes.c_int32), ("U_override", ctypes.c_int32),
         ("idx_cols", ctypes.c_int32), ("idx_per_head", ctypes.c_int32),
         ("path", ctypes.c_int32), ("idx_shared", ctypes.c_int32), ("c", ctypes.c_double),
+        ("r_sparse", ctypes.c_double),
         ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
         ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3),
     ]
@@ -83,6 +85,7 @@ def load(build_if_missing: bool = True):
     lib.psattn_plan_enable_host_io.argtypes = [vp]
     lib.psattn_forward_host.argtypes = [vp] * 9
     lib.psattn_mean_v_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.psattn_probe_gather.argtypes = [i32, vp, ctypes.c_int64, i32, i32, i32, vp, vp]
     _lib = lib
     return lib
 
@@ -128,12 +131,21 @@ def psattn_mean_v_noalloc(V, lengths, vbar, B, H, T_max):
     return vbar
 
 
+def psattn_probe_gather(mode, rows, n_ctas, warps_per_cta, rounds_per_warp, sink):
+    """Launches the gather microbenchmark (see include/psattn.h); returns the number of 128-byte rows it reads."""
+    n_rows = 0 if rows is None else rows.numel() * rows.element_size() // 128
+    _check(load().psattn_probe_gather(int(mode), _ptr(rows), n_rows, int(n_ctas), int(warps_per_cta),
+                                      int(rounds_per_warp), _ptr(sink), _stream()))
+    per = {0: 1, 1: 2, 2: 4}[int(mode)]
+    return int(n_ctas) * int(warps_per_cta) * (int(rounds_per_warp) // per * per) * 16
+
+
 class Plan:
     """Owns a psattn_plan_t and a zero-initialised workspace tensor on the current device."""
 
     def __init__(self, B, H, T_max, dtype=torch.bfloat16, c=5.0, idx_cols=None, d_head=64,
                  fill_mode=PSATTN_FILL_MEAN_V, u_override=0, U_override=0, idx_per_head=False,
-                 path=PSATTN_PATH_AUTO, strides=None, idx_shared=False):
+                 path=PSATTN_PATH_AUTO, strides=None, idx_shared=False, r_sparse=0.0):
         lib = load()
         self.lib = lib
         d = psattn_desc_t()
@@ -145,6 +157,7 @@ class Plan:
                 [psattn_count(c, L) for L in range(1, T_max + 1)] + [1])
         d.idx_cols, d.idx_per_head, d.path, d.c = idx_cols, int(idx_per_head), path, c
         d.idx_shared = int(idx_shared)
+        d.r_sparse = float(r_sparse)
         if strides is not None:
             for name in ("q", "k", "v", "o"):
                 if name in strides:

@@ -98,6 +98,7 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     if (d.u_override < 0 || d.U_override < 0 || d.idx_cols < 1) return PSATTN_ERR_BAD_DESC;
     if (d.idx_shared != 0 && d.idx_shared != 1) return PSATTN_ERR_BAD_DESC;
     if (!(d.c > 0.0) || !std::isfinite(d.c)) return PSATTN_ERR_BAD_DESC;
+    if (!(d.r_sparse >= 0.0) || d.r_sparse > 1.0) return PSATTN_ERR_BAD_DESC;
     if (d.d_head != kD) return PSATTN_ERR_UNSUPPORTED;
     int rc;
     if ((rc = check_strides(d.q_stride, d)) || (rc = check_strides(d.k_stride, d)) ||
@@ -110,6 +111,12 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     for (int len = 0; len <= d.T_max; ++len) {
         int n = psattn_count(d.c, len);
         int u = d.u_override > 0 ? (d.u_override < len ? d.u_override : len) : n;
+        if (d.r_sparse > 0.0 && len > 0) {      // Sec. 3.2: L_sparse = r_sparse L, from the sequence's own length
+            double x = std::ceil(d.r_sparse * (double)len);
+            if (x < 1.0) x = 1.0;
+            if (x > (double)len) x = (double)len;
+            u = (int)x;
+        }
         int U = d.U_override > 0 ? (len > 0 ? d.U_override : 0) : n;
         if (U > d.idx_cols) {
             if (d.U_override > 0) U = d.idx_cols;
@@ -205,7 +212,16 @@ extern "C" int psattn_workspace_bytes(const psattn_plan_t *p, size_t *bytes) {
 // ---- helpers ---------------------------------------------------------------------------
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// A plan belongs to the device that was current when it was created: its tables, its streams and the
+// kernels' shared-memory grants live there.
+static int check_device(const psattn_plan_t *p) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return PSATTN_ERR_NO_DEVICE; }
+    return dev == p->device ? PSATTN_OK : PSATTN_ERR_BAD_DESC;
+}
+
 static int check_ws(const psattn_plan_t *p, const void *ws, size_t bytes) {
+    if (int rc = check_device(p)) return rc;
     if (!ws) return PSATTN_ERR_NULL;
     if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return PSATTN_ERR_MISALIGNED;
     if (bytes < p->ws_bytes) return PSATTN_ERR_WORKSPACE_TOO_SMALL;
@@ -279,7 +295,7 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
     if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && rows != nullptr && n_rows + (vbar ? 1 : 0) <= 64) {
         // one CTA per SM: split the keys only when there are fewer units than SMs
         const int pairs = (d.T_max + 255) / 256;
-        int splits = 148 / (d.B * d.H > 0 ? d.B * d.H : 1);
+        int splits = device_sm_count() / (d.B * d.H > 0 ? d.B * d.H : 1);
         if (splits > plan->n_splits) splits = plan->n_splits;
         if (splits > pairs) splits = pairs;
         if (splits < 1) splits = 1;
@@ -299,7 +315,7 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
         // key splits: enough CTAs to cover the SMs about twice, never more splits than 128-key tiles
         const int tiles = (d.T_max + 127) / 128;
         const long long ctas = (long long)d.B * d.H * ((n_rows + 127) / 128);
-        int splits = (int)((2 * 148 + ctas - 1) / (ctas > 0 ? ctas : 1));
+        int splits = (int)((2 * device_sm_count() + ctas - 1) / (ctas > 0 ? ctas : 1));
         if (splits > plan->n_splits) splits = plan->n_splits;
         if (splits > tiles) splits = tiles;
         if (splits < 1 || rows == nullptr) splits = 1;
@@ -412,7 +428,7 @@ extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
-    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && d.B * d.H >= kSmCount / 2) {
+    if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED && d.B * d.H >= device_sm_count() / 2) {
         // one kernel for steps (d)+(e), one CTA per unit: where the units cover at least half of the SMs
         cudaError_t e = launch_forward_fused(g, plan->U_max, d.fill_mode == PSATTN_FILL_OWN_V, Q, K, V, nullptr, O,
                                              nullptr, nullptr, sel_idx_in, st);
@@ -531,6 +547,7 @@ extern "C" int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const vo
 extern "C" int psattn_read_status(psattn_plan_t *plan, void *workspace, void *stream,
                                   uint32_t *host_bits) {
     if (!plan || !workspace || !host_bits) return PSATTN_ERR_NULL;
+    if (int rc = check_device(plan)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned *w = ws_at<unsigned>(workspace, plan->off_status);
     PSATTN_CU(cudaMemcpyAsync(host_bits, w, sizeof(unsigned), cudaMemcpyDeviceToHost, st));
@@ -542,6 +559,7 @@ extern "C" int psattn_read_status(psattn_plan_t *plan, void *workspace, void *st
 // ---- host-buffer front end ------------------------------------------------------------------
 extern "C" int psattn_plan_enable_host_io(psattn_plan_t *plan) {
     if (!plan) return PSATTN_ERR_NULL;
+    if (int rc = check_device(plan)) return rc;
     if (plan->host_io) return PSATTN_OK;
     const psattn_desc_t &d = plan->desc;
     const size_t es = d.dtype == PSATTN_BF16 ? 2 : 4;
@@ -571,6 +589,7 @@ extern "C" int psattn_forward_host(psattn_plan_t *plan, const void *Q, const voi
                                    int32_t *sel_idx, void *stream) {
     if (!plan || !Q || !K || !V || !sample_idx || !O || !sel_idx) return PSATTN_ERR_NULL;
     if (!plan->host_io) return PSATTN_ERR_BAD_DESC;
+    if (int rc = check_device(plan)) return rc;
     psattn_desc_t &d = plan->desc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t es = d.dtype == PSATTN_BF16 ? 2 : 4;

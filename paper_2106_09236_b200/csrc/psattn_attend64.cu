@@ -33,13 +33,16 @@ __global__ void __launch_bounds__(kA64Threads, 1) k_attend64(Geom g, Attend64Arg
         if (tid == 0) atomicOr(g.status, kStatusWaitExpired);
         return;
     }
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // programmatic dependent launch, see pdl_enter
     if (warp == 0) tmem_alloc(tmem_slot_p, kA64TmemCols);
     if (tid == 32) { tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_p;
+    // Programmatic dependent launch (see pdl_enter), only now that this CTA holds its TMEM: a dependent CTA
+    // that starts early allocates TMEM too and then sits in its griddepcontrol.wait; if it could take the
+    // columns before a CTA of this grid had allocated, that CTA would block in tcgen05.alloc for good.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");                // nothing above touches global data
 
     Attend64Job j;
@@ -126,6 +129,7 @@ cudaError_t launch_attend64(const Geom &g, const void *Q, const void *K, const v
                             int out_by_position, int out_fp32, float *vbar, cudaStream_t st) {
     if (g.B * g.H == 0 || n_rows == 0) return cudaSuccess;
     if (n_rows + (vbar ? 1 : 0) > kA64MaxRows || rows == nullptr || (split_keys % 256) != 0) return cudaErrorNotSupported;
+    if ((long long)g.B * g.H > 65535) return cudaErrorNotSupported;         // the unit index is gridDim.y
     Attend64Args a;
     a.rows = rows; a.n_rows = n_rows; a.rows_stride = rows_stride;
     a.n_splits = n_splits; a.split_keys = split_keys;
@@ -138,12 +142,8 @@ cudaError_t launch_attend64(const Geom &g, const void *Q, const void *K, const v
         return cudaErrorNotSupported;
     if (posK[0] != posV[0] || posK[1] != posV[1] || posK[2] != posV[2]) return cudaErrorNotSupported;
     a.pos_t = posK[0]; a.pos_h = posK[1]; a.pos_b = posK[2];
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_attend64, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kA64Bytes);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_attend64, grant, kA64Bytes)) return e;
     dim3 grid((unsigned)n_splits, (unsigned)(g.B * g.H));
     cudaError_t le = launch_pdl(k_attend64, grid, dim3(kA64Threads), kA64Bytes, st, g, a, (const __nv_bfloat16 *)Q, tmK, tmV);
     if (le != cudaSuccess) { note_launch(); return le; }

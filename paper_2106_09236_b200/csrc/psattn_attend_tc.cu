@@ -329,6 +329,7 @@ cudaError_t launch_attend_tc(const Geom &g, const void *Q, const void *K, const 
                              float *part_acc, void *out, long long out_unit_stride, long long out_row_stride,
                              int out_by_position, int out_fp32, cudaStream_t st) {
     if (g.B * g.H == 0 || n_rows == 0) return cudaSuccess;
+    if ((long long)g.B * g.H > 65535 || (n_rows + kTileRows - 1) / kTileRows > 65535) return cudaErrorNotSupported;   // gridDim.z, .y
     AttendTcArgs a;
     a.rows = rows; a.n_rows = n_rows; a.rows_stride = rows_stride;
     a.n_splits = n_splits; a.split_keys = split_keys;
@@ -340,16 +341,9 @@ cudaError_t launch_attend_tc(const Geom &g, const void *Q, const void *K, const 
     if (!make_kv_map(&tmK, K, g, g.ks, posK) || !make_kv_map(&tmV, V, g, g.vs, posV)) return cudaErrorNotSupported;
     if (posK[0] != posV[0] || posK[1] != posV[1] || posK[2] != posV[2]) return cudaErrorNotSupported;
     a.pos_t = posK[0]; a.pos_h = posK[1]; a.pos_b = posK[2];
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttendSmem);
-        // two CTAs fit an SM (2 x 113 KB of shared memory, 2 x 256 TMEM columns) and hide each other's waits
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k_attend_tc, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                     cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    // two CTAs fit an SM (2 x 113 KB of shared memory, 2 x 256 TMEM columns) and hide each other's waits
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_attend_tc, grant, kAttendSmem, true)) return e;
     dim3 grid((unsigned)n_splits, (unsigned)((n_rows + kTileRows - 1) / kTileRows), (unsigned)(g.B * g.H));
     k_attend_tc<<<grid, 128, kAttendSmem, st>>>(g, a, (const __nv_bfloat16 *)Q, tmK, tmV);
     note_launch();

@@ -189,12 +189,8 @@ cudaError_t launch_exact_measure(int dtype, const Geom &g, const void *Q, const 
         int pq[3], pk[3];
         if (make_rows_map(&tmQ, Q, g, g.qs, kEmRows, 1, pq) && make_rows_map(&tmK, K, g, g.ks, kEmKeys, 1, pk) &&
             pq[0] == pk[0] && pq[1] == pk[1] && pq[2] == pk[2]) {
-            static bool attr_set = false;
-            if (!attr_set) {
-                cudaError_t e = cudaFuncSetAttribute(k_exact_measure, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kEmSmem);
-                if (e != cudaSuccess) return e;
-                attr_set = true;
-            }
+            static SmemGrant grant;
+            if (cudaError_t e = grant_dynamic_smem(k_exact_measure, grant, kEmSmem)) return e;
             const dim3 grid((unsigned)units, (unsigned)((g.T + kEmRows - 1) / kEmRows));
             k_exact_measure<<<grid, kEmRows, kEmSmem, st>>>(g, pq[0], pq[1], pq[2], M, tmQ, tmK);
             note_launch();

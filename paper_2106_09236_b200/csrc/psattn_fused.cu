@@ -60,7 +60,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     // wait at their own griddepcontrol.wait until this grid has completed and its writes are visible),
     // and do not touch global memory before the previous grid has completed.  Both are no-ops when the
     // launch carries no programmatic dependency.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // The trigger comes after this CTA's TMEM allocation (below, behind the barrier that publishes the slot):
+    // a dependent CTA allocates TMEM and then waits for this grid, so it must never get columns that a CTA
+    // of this grid still needs.
     if (warp == 0) tmem_alloc(&P.tmem_slot, kA64TmemCols);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // Which unit this CTA works on.  With ragged lengths the CTAs take the sequences longest first
@@ -99,6 +101,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = P.tmem_slot;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- steps (a)+(b) ------------------------------------------------------------------------
     bool ok = true;
@@ -212,13 +215,9 @@ cudaError_t launch_forward_fused(const Geom &g, int U_max, int own_v, const void
     a.own_v = own_v;
     a.sel_in = sel_in;
     // the ranking costs B comparisons per sequence in every CTA: only where a second wave exists and B is small
-    a.by_length = g.lengths != nullptr && g.B * g.H > kSmCount && g.B <= 256;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(k_forward_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_smem = smem;
-    }
+    a.by_length = g.lengths != nullptr && g.B * g.H > device_sm_count() && g.B <= 256;
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_forward_fused, grant, smem)) return e;
     // launched with programmatic stream serialization: the kernel may be scheduled while the previous
     // kernel of the stream drains; it orders itself with griddepcontrol.wait before its first read
     cudaLaunchConfig_t cfg = {};

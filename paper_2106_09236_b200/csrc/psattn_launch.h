@@ -8,8 +8,23 @@ constexpr int kColsumRows = 256;      // rows of V per column-sum partial
 constexpr int kFillRows = 128;        // rows of O per fill block
 constexpr int kSelectThreads = 1024;
 constexpr int kSelectSmemKeys = 8192; // keys kept in shared memory by the select kernel (32 KB)
-constexpr int kSmCount = 148;         // SMs of a B200
 constexpr int kSplitKeys = 1024;      // keys per split of the SIMT attention kernel
+constexpr int kMaxDevices = 64;       // device ordinals the per-device records below cover
+
+// Multiprocessors of the current device (read once per device from its attributes).
+int device_sm_count();
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to the current device's context: one record per
+// kernel holds, per device, the size already granted there.  grant_dynamic_smem raises it when needed
+// (thread safe; `carveout`: also ask for the largest shared-memory carve-out).
+struct SmemGrant {
+    size_t bytes[kMaxDevices];
+};
+cudaError_t grant_dynamic_smem_impl(const void *kernel, SmemGrant &rec, size_t smem, bool carveout);
+template <typename... KArgs>
+inline cudaError_t grant_dynamic_smem(void (*kernel)(KArgs...), SmemGrant &rec, size_t smem, bool carveout = false) {
+    return grant_dynamic_smem_impl(reinterpret_cast<const void *>(kernel), rec, smem, carveout);
+}
 
 // Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in the
 // stream drains.  Only for kernels that call pdl_enter() before their first global-memory access.

@@ -133,16 +133,12 @@ cudaError_t launch_measure_mma(const Geom &g, int U_max, const void *Q, const vo
     const int units = g.B * g.H;
     // resident CTAs per SM by shared memory; slices so that the grid covers the SMs
     const int per_sm = smem <= 100 * 1024 ? 2 : 1;
-    int slices = (148 * per_sm) / units;
+    int slices = (device_sm_count() * per_sm) / units;
     if (slices < 1) slices = 1;
     if (slices > 8) slices = 8;
     a.q_slices = slices;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(k_measure_mma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_smem = smem;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_measure_mma, grant, smem)) return e;
     k_measure_mma<<<(unsigned)(units * slices), kMeasureThreads, smem, st>>>(g, a, (const __nv_bfloat16 *)Q, sidx, M, tmK);
     note_launch();
     return cudaGetLastError();
@@ -164,15 +160,11 @@ cudaError_t launch_measure_stream(const Geom &g, int U_max, const void *Q, const
     const int units = g.B * g.H;
     constexpr int kBlock = measure_block_queries(kStreamThreads);
     const int blocks_total = (g.T + kBlock - 1) / kBlock;
-    int slices = (2 * 148 + units - 1) / units;             // about two CTAs' worth of work per SM
+    int slices = (2 * device_sm_count() + units - 1) / units;             // about two CTAs' worth of work per SM
     if (slices > blocks_total) slices = blocks_total;
     if (slices < 1) slices = 1;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        cudaError_t e = cudaFuncSetAttribute(k_measure_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_smem = smem;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_measure_stream, grant, smem)) return e;
     cudaError_t e = launch_pdl(k_measure_stream, dim3((unsigned)(units * slices)), dim3(kStreamThreads), smem, st, g, slices,
                                (uint32_t)stage_bytes, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, sidx, M);
     note_launch();

@@ -1,5 +1,5 @@
 // Steps (a)+(b) (Eq. 11) when one sample of keys serves every query of a sequence (the other reading of
-// "a random sampling key matrix" in Sec. 3.2): the sampled scores of a tile of queries are then one dense
+// how Sec. 3.2 draws the sampled keys): the sampled scores of a tile of queries are then one dense
 // product Q_tile K~^T, which belongs on the tensor cores.
 //
 // One CTA = (unit, run of 128-query tiles), 128 threads:
@@ -155,17 +155,13 @@ cudaError_t launch_measure_shared(const Geom &g, int U_max, const void *Q, const
     if (!make_rows_map(&tmQ, Q, g, g.qs, kMsRows, 1, pos)) return cudaErrorNotSupported;
     // runs of tiles long enough to amortise the gather of the sampled keys, short enough for a few CTAs per SM
     const int units = g.B * g.H, tiles_total = (g.T + kMsRows - 1) / kMsRows;
-    int chunks = (4 * kSmCount + units - 1) / units;
+    int chunks = (4 * device_sm_count() + units - 1) / units;
     if (chunks > tiles_total) chunks = tiles_total;
     if (chunks < 1) chunks = 1;
     const int tiles_per_cta = (tiles_total + chunks - 1) / chunks;
     chunks = (tiles_total + tiles_per_cta - 1) / tiles_per_cta;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_measure_shared, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMsSmem);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_measure_shared, grant, kMsSmem)) return e;
     const dim3 grid((unsigned)units, (unsigned)chunks);
     k_measure_shared<<<grid, kMsRows, kMsSmem, st>>>(g, tiles_per_cta, pos[0], pos[1], pos[2], (const __nv_bfloat16 *)K,
                                                       sidx, M, tmQ);

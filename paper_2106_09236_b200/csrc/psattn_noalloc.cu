@@ -34,7 +34,6 @@ __global__ void __launch_bounds__(kD) k_mean_finish(Geom g, const float *__restr
     vbar[(long long)unit * kD + threadIdx.x] = L > 0 ? s / (float)L : 0.f;
 }
 
-constexpr int kMaxDevices = 64;
 static std::mutex g_setup_mutex;
 static float *g_scratch_addr[kMaxDevices];          // device address of the array, per device
 
@@ -62,7 +61,7 @@ extern "C" int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, floa
                                      int32_t B, int32_t H, int32_t T_max, int32_t dtype,
                                      void *stream) {
     if (!V || !vbar) return PSATTN_ERR_NULL;
-    if (B < 0 || H < 1 || T_max < 1) return PSATTN_ERR_BAD_DESC;
+    if (B < 0 || H < 1 || T_max < 1 || B > (1 << 20) || H > 4096 || T_max > (1 << 20)) return PSATTN_ERR_BAD_DESC;
     if (dtype != PSATTN_BF16 && dtype != PSATTN_FP32) return PSATTN_ERR_BAD_DESC;
     if ((reinterpret_cast<uintptr_t>(V) & 15u) != 0) return PSATTN_ERR_MISALIGNED;
     const long long units = (long long)B * H;

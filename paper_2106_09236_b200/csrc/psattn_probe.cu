@@ -1,0 +1,197 @@
+// Microbenchmarks of the two gather rates that bound steps (a)+(b) (Eq. 11): every (query, sampled key)
+// pair needs one 128-byte key row, read at a random position
+//   mode 0  out of shared memory (keys of a unit resident: T_max <= ~1100), with the ldmatrix access
+//           pattern of psattn_measure_mma.cuh (16 rows per round, rotated 16-byte chunks);
+//   mode 1  out of L2 into registers (longer sequences), with the access pattern of
+//           psattn_measure_stream.cuh (16 rows per round, four 16-byte loads per lane).
+// Nothing is computed: the loaded words are xor-ed into a sink so that the loads stay.  The benchmark
+// times these kernels with CUDA events and reports the measure kernels against the rates found.
+#include "../../include/psattn.h"
+
+#include "psattn_launch.h"
+#include "psattn_sm100.cuh"
+
+namespace psattn {
+
+constexpr int kProbeSmemRows = 1024;                       // 128 KB of 128-byte rows
+
+__device__ __forceinline__ uint32_t probe_hash(uint32_t x) {
+    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+    return x;
+}
+
+__global__ void __launch_bounds__(1024, 1) k_probe_smem(int rounds, uint32_t *__restrict__ sink) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int e = tid; e < kProbeSmemRows * 32; e += blockDim.x) reinterpret_cast<uint32_t *>(smem)[e] = (uint32_t)e;
+    __syncthreads();
+    const uint32_t base = sm100::smem_u32(smem);
+    const int l7 = lane & 7;
+    uint32_t off[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) off[t] = (uint32_t)((2 * t + (lane >> 4) + l7) & 7) << 4;
+    uint32_t acc = 0;
+    uint32_t seed = (blockIdx.x * 64u + warp) * 65536u;
+#pragma unroll 2
+    for (int r = 0; r < rounds; ++r) {
+        // lane l addresses row (l & 7) + 8 * ((l >> 3) & 1) of the round: a random key of the resident chunk
+        const uint32_t row = probe_hash(seed + (uint32_t)r * 16u + (uint32_t)(l7 + 8 * ((lane >> 3) & 1))) % kProbeSmemRows;
+        const uint32_t ra = base + row * 128u;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            uint32_t a0, a1, a2, a3;
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3)
+                         : "r"(ra + off[t]));
+            acc ^= a0 ^ a1 ^ a2 ^ a3;
+        }
+    }
+    if (acc == 0x12345678u) sink[0] = acc;                 // practically never: keeps the loads alive
+}
+
+// Same gather with the arithmetic of the measure kernel behind it: the four ldmatrix tiles of a round feed a
+// chain of four mma.m16n8k16; kChains rounds are interleaved.  kIdx: the row numbers come from a table in
+// shared memory (one 4-byte load per lane and round) instead of a hash.
+template <int kChains, bool kIdx>
+__global__ void __launch_bounds__(1024, 1) k_probe_smem_mma(int rounds, uint32_t *__restrict__ sink) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int e = tid; e < kProbeSmemRows * 32; e += blockDim.x) reinterpret_cast<uint32_t *>(smem)[e] = (uint32_t)e;
+    uint32_t *table = reinterpret_cast<uint32_t *>(smem + kProbeSmemRows * 128);        // 4096 row numbers
+    for (int e = tid; e < 4096; e += blockDim.x) table[e] = probe_hash((uint32_t)e * 7919u + blockIdx.x) % kProbeSmemRows;
+    __syncthreads();
+    const uint32_t base = sm100::smem_u32(smem), tbase = sm100::smem_u32(table);
+    const int l7 = lane & 7;
+    uint32_t off[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) off[t] = (uint32_t)((2 * t + (lane >> 4) + l7) & 7) << 4;
+    uint32_t bq[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) bq[t] = 0x3f803f80u + (uint32_t)(lane + t);
+    float mx = 0.f, ds = 0.f;
+    const uint32_t seed = (blockIdx.x * 64u + warp) * 65536u;
+    const uint32_t slot = (uint32_t)(l7 + 8 * ((lane >> 3) & 1));
+    for (int r = 0; r + kChains <= rounds; r += kChains) {
+        float c[kChains][4];
+        uint32_t ra[kChains];
+#pragma unroll
+        for (int k = 0; k < kChains; ++k) {
+            uint32_t row;
+            if (kIdx) {
+                const uint32_t ta = tbase + ((((uint32_t)(r + k) * 16u + slot + (uint32_t)warp * 64u) & 4095u) << 2);
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(row) : "r"(ta));
+            } else {
+                row = probe_hash(seed + (uint32_t)(r + k) * 16u + slot) % kProbeSmemRows;
+            }
+            ra[k] = base + row * 128u;
+        }
+#pragma unroll
+        for (int k = 0; k < kChains; ++k) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                uint32_t a0, a1, a2, a3;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3)
+                             : "r"(ra[k] + off[t]));
+                if (t == 0)
+                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%10, %10, %10, %10};"
+                                 : "=f"(c[k][0]), "=f"(c[k][1]), "=f"(c[k][2]), "=f"(c[k][3])
+                                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bq[0]), "r"(bq[1]), "f"(0.f));
+                else
+                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                                 : "+f"(c[k][0]), "+f"(c[k][1]), "+f"(c[k][2]), "+f"(c[k][3])
+                                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bq[2 * t]), "r"(bq[2 * t + 1]));
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kChains; ++k) {
+            mx = fmaxf(mx, fmaxf(c[k][0], c[k][2]));
+            ds += c[k][1] + c[k][3];
+        }
+    }
+    if (mx + ds == 0.12345f) sink[0] = 1u;
+}
+
+template <int kInFlight>
+__global__ void __launch_bounds__(768, 1) k_probe_l2(const uint4 *__restrict__ rows, uint32_t n_rows, int rounds,
+                                                     uint32_t *__restrict__ sink) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    uint32_t acc = 0;
+    const uint32_t seed = (blockIdx.x * 64u + warp) * 65536u;
+    for (int r0 = 0; r0 < rounds; r0 += kInFlight) {
+        uint4 v[kInFlight][4];
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k) {
+            // rows g and g + 8 of the round; lanes t = 0..3 read the four 16-byte pieces of each half row
+            const uint32_t ra = probe_hash(seed + (uint32_t)(r0 + k) * 16u + (uint32_t)g) % n_rows;
+            const uint32_t rb = probe_hash(seed + (uint32_t)(r0 + k) * 16u + (uint32_t)(g + 8)) % n_rows;
+            const uint4 *pa = rows + (size_t)ra * 8 + t, *pb = rows + (size_t)rb * 8 + t;
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(v[k][0].x), "=r"(v[k][0].y), "=r"(v[k][0].z), "=r"(v[k][0].w) : "l"(pa));
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(v[k][1].x), "=r"(v[k][1].y), "=r"(v[k][1].z), "=r"(v[k][1].w) : "l"(pa + 4));
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(v[k][2].x), "=r"(v[k][2].y), "=r"(v[k][2].z), "=r"(v[k][2].w) : "l"(pb));
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(v[k][3].x), "=r"(v[k][3].y), "=r"(v[k][3].z), "=r"(v[k][3].w) : "l"(pb + 4));
+        }
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) acc ^= v[k][x].x ^ v[k][x].y ^ v[k][x].z ^ v[k][x].w;
+    }
+    if (acc == 0x12345678u) sink[0] = acc;
+}
+
+}  // namespace psattn
+
+using namespace psattn;
+
+extern "C" int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_rows, int32_t n_ctas,
+                                   int32_t warps_per_cta, int32_t rounds_per_warp, uint32_t *sink,
+                                   void *stream) {
+    if (!sink) return PSATTN_ERR_NULL;
+    if (n_ctas < 1 || n_ctas > 65535 || rounds_per_warp < 1 || warps_per_cta < 1) return PSATTN_ERR_BAD_DESC;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (mode == 0) {
+        if (warps_per_cta > 32) return PSATTN_ERR_BAD_DESC;
+        static SmemGrant grant;
+        const size_t smem = (size_t)kProbeSmemRows * 128;
+        if (grant_dynamic_smem(k_probe_smem, grant, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+        k_probe_smem<<<(unsigned)n_ctas, (unsigned)warps_per_cta * 32, smem, st>>>(rounds_per_warp, sink);
+    } else if (mode >= 3 && mode <= 8) {
+        if (warps_per_cta > 32) return PSATTN_ERR_BAD_DESC;
+        const size_t smem = (size_t)kProbeSmemRows * 128 + 4096 * 4;
+        static SmemGrant g3, g4, g5, g6, g7, g8;
+        const dim3 grid((unsigned)n_ctas), block((unsigned)warps_per_cta * 32);
+#define PSATTN_PROBE_CASE(M, G, CH, IDX)                                                                   \
+        case M:                                                                                            \
+            if (grant_dynamic_smem(k_probe_smem_mma<CH, IDX>, G, smem) != cudaSuccess) return PSATTN_ERR_CUDA; \
+            k_probe_smem_mma<CH, IDX><<<grid, block, smem, st>>>(rounds_per_warp, sink);                   \
+            break;
+        switch (mode) {
+            PSATTN_PROBE_CASE(3, g3, 1, false)
+            PSATTN_PROBE_CASE(4, g4, 2, false)
+            PSATTN_PROBE_CASE(5, g5, 4, false)
+            PSATTN_PROBE_CASE(6, g6, 1, true)
+            PSATTN_PROBE_CASE(7, g7, 2, true)
+            PSATTN_PROBE_CASE(8, g8, 4, true)
+        }
+#undef PSATTN_PROBE_CASE
+    } else if (mode == 1 || mode == 2) {
+        if (!rows) return PSATTN_ERR_NULL;
+        if (n_rows < 1 || n_rows > (1ll << 31) || warps_per_cta > 24) return PSATTN_ERR_BAD_DESC;
+        if ((reinterpret_cast<uintptr_t>(rows) & 15u) != 0) return PSATTN_ERR_MISALIGNED;
+        if (mode == 1)
+            k_probe_l2<2><<<(unsigned)n_ctas, (unsigned)warps_per_cta * 32, 0, st>>>((const uint4 *)rows, (uint32_t)n_rows,
+                                                                                  rounds_per_warp / 2 * 2, sink);
+        else
+            k_probe_l2<4><<<(unsigned)n_ctas, (unsigned)warps_per_cta * 32, 0, st>>>((const uint4 *)rows, (uint32_t)n_rows,
+                                                                                  rounds_per_warp / 4 * 4, sink);
+    } else {
+        return PSATTN_ERR_BAD_DESC;
+    }
+    note_launch();
+    return cudaGetLastError() == cudaSuccess ? PSATTN_OK : PSATTN_ERR_CUDA;
+}

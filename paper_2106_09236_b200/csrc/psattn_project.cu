@@ -80,11 +80,13 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
     __syncwarp();
     // programmatic dependent launch: the next kernel of the stream may be scheduled now (it waits at its own
     // griddepcontrol.wait); nothing in global memory is touched before the previous grid has completed
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // (the trigger comes after this CTA's TMEM allocation: a dependent CTA that allocates TMEM and then waits
+    // for this grid must never get the columns a CTA of this grid still needs)
     if (warp == 1) tmem_alloc(tmem_slot, 512);                 // two accumulators, 192 of 256 columns each
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     const int n_kb = (a.dx + kPjK - 1) / kPjK;
@@ -346,18 +348,14 @@ cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
         if (ok) {
-            static bool attr_set = false;
-            if (!attr_set) {
-                cudaError_t e = cudaFuncSetAttribute(k_project_qkv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPjSmem);
-                if (e != cudaSuccess) return e;
-                attr_set = true;
-            }
+            static SmemGrant grant;
+            if (cudaError_t e = grant_dynamic_smem(k_project_qkv, grant, kPjSmem)) return e;
             // both kernels carry a programmatic dependency on their predecessor in the stream
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
             attr[0].val.programmaticStreamSerializationAllowed = 1;
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)(a.n_tiles < kSmCount ? a.n_tiles : kSmCount));
+            cfg.gridDim = dim3((unsigned)(a.n_tiles < device_sm_count() ? a.n_tiles : device_sm_count()));
             cfg.blockDim = dim3(kPjThreads);
             cfg.dynamicSmemBytes = kPjSmem;
             cfg.stream = st;

@@ -7,6 +7,7 @@
 #include "psattn_select.cuh"
 
 #include <atomic>
+#include <mutex>
 
 namespace psattn {
 
@@ -404,6 +405,35 @@ __global__ void __launch_bounds__(256) k_fill(Geom g, const DT *__restrict__ V,
 // Host-side launchers
 // ---------------------------------------------------------------------------------------
 static std::atomic<unsigned long long> g_launches{0};
+int device_sm_count() {
+    static std::atomic<int> cached[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 1; }
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    int n = slot ? cached[dev].load(std::memory_order_relaxed) : 0;
+    if (n <= 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { cudaGetLastError(); n = 1; }
+        if (slot) cached[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+
+cudaError_t grant_dynamic_smem_impl(const void *kernel, SmemGrant &rec, size_t smem, bool carveout) {
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool slot = dev >= 0 && dev < kMaxDevices;
+    std::lock_guard<std::mutex> lock(mu);
+    if (slot && rec.bytes[dev] >= smem) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess && carveout)
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    if (slot) rec.bytes[dev] = smem;
+    return cudaSuccess;
+}
+
 void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
 
@@ -440,7 +470,7 @@ cudaError_t launch_select(const Geom &g, const float *M, int *sel, const float *
                           float *vbar, int *cand, cudaStream_t st) {
     if (g.B * g.H == 0) return cudaSuccess;
     const int units = g.B * g.H;
-    int slices = kSmCount / units;
+    int slices = device_sm_count() / units;
     if (slices > kSelectMaxSlices) slices = kSelectMaxSlices;
     if (M != nullptr && vbar == nullptr && cand != nullptr && slices >= 2 && g.u_max <= 64 && g.T / slices >= 1024) {
         const int width = (g.T + slices - 1) / slices;

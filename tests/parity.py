@@ -89,10 +89,10 @@ def check_outputs(O_gpu, O_ref, swaps, inp, lengths, dtype, fill="mean_v"):
 
 
 def check_forward(O_gpu, sel_gpu, M_gpu, inp, lengths, dtype, c, u_override=0, U_override=0,
-                  fill="mean_v", nthreads=8):
+                  fill="mean_v", nthreads=8, r_sparse=0.0):
     O_ref, sel_ref, M_ref = orc.forward(inp["Q"], inp["K"], inp["V"], inp["sample_idx"], lengths,
                                         c=c, u_override=u_override, U_override=U_override,
-                                        fill=fill, nthreads=nthreads)
+                                        fill=fill, nthreads=nthreads, r_sparse=r_sparse)
     if M_gpu is not None:
         check_measure(M_gpu, M_ref, lengths)
     w = sel_ref.shape[-1]

@@ -60,7 +60,8 @@ def test_plan_create_rejects_bad_descriptors_before_touching_a_device():
 
     assert lib.psattn_plan_create(None, ctypes.byref(h)) == 1
     for bad in (dict(H=0), dict(T_max=0), dict(dtype=5), dict(fill_mode=9), dict(c=0.0),
-                dict(c=float("nan")), dict(idx_cols=0), dict(path=7), dict(u_override=-1)):
+                dict(c=float("nan")), dict(idx_cols=0), dict(path=7), dict(u_override=-1),
+                dict(r_sparse=-0.1), dict(r_sparse=1.5), dict(r_sparse=float("nan"))):
         assert lib.psattn_plan_create(ctypes.byref(make(**bad)), ctypes.byref(h)) == 2, bad
         assert h.value is None
     assert lib.psattn_plan_create(ctypes.byref(make(d_head=128)), ctypes.byref(h)) == 3

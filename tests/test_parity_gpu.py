@@ -161,6 +161,25 @@ def test_paper_literal_variant_at_scale(dtype, T, r_sparse):
     parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c, u_override=u, fill="own_v")
 
 
+@pytest.mark.parametrize("r_sparse", [0.35, 0.5])
+@pytest.mark.parametrize("dtype,T", [("bf16", 500), ("bf16", 1400), ("fp32", 160)])
+def test_paper_count_rule_per_sequence(dtype, T, r_sparse):
+    """Sec. 3.2 as stated: L_sparse = r_sparse L from every sequence's OWN length (descriptor field
+    r_sparse), ragged batch, Eq. 12's v_i fill; r_sample = 1 (c = 1) as in the paper's timed model."""
+    H, c = 4, 1.0
+    rng = np.random.default_rng(900 + T)
+    lengths = [T, 1, 40] + [int(x) for x in rng.integers(40, T + 1, size=5)]
+    n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+    inp = _synth(len(lengths), H, T, 147 + T, n_cols, dtype, lengths)
+    O, sel, M, status = _run_forward(inp, dtype, c, ps.PSATTN_PATH_AUTO, r_sparse=r_sparse,
+                                     fill_mode=ps.PSATTN_FILL_OWN_V)
+    assert status == 0
+    assert sel.shape[-1] == int(np.ceil(r_sparse * T))
+    for b, L in enumerate(lengths):
+        assert int((sel[b, 0] >= 0).sum()) == max(1, int(np.ceil(r_sparse * L)))
+    parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c, fill="own_v", r_sparse=r_sparse)
+
+
 @pytest.mark.parametrize("T", [80, 1300])           # keys resident in shared memory / streamed from L2
 @pytest.mark.parametrize("path", PATHS, ids=PATH_IDS)
 def test_out_of_range_inputs_set_status_bits_without_faulting(path, T):

@@ -14,6 +14,7 @@
  *   Eq. 11    its sampled approximation          M~ = max - mean over K~
  *   Eq. 12    the piecewise output (attention for I_sparse, cheap value else)
  *   Sec. 3.2  the sample size  L~ = r_sample * ln L  and the top-L_sparse rule
+ *   Sec. 2.2 / 3.1  the output matrix that merges the heads after the attention
  *
  * Readings taken where the paper is silent or garbled (kept in one place so a
  * reader can check them):
@@ -340,6 +341,36 @@ void psattn_oracle_project_qkv(const float *X, const float *Wt, int B, int T, in
                         for (int k = 0; k < dx; ++k) acc += (double)x[k] * (double)w[k];
                     out[r * plane + (((size_t)b * H + h) * T + t) * d + e] = acc;
                 }
+    }
+}
+
+/*
+ * The output side of the attention module (Sec. 2.2, Eq. 5 places MHSA inside the Conformer block;
+ * Sec. 3.1 defines its heads): the heads' outputs are concatenated and multiplied by one output matrix,
+ *   Y[b][t][n] = sum_h sum_e O[b][h][t][e] * W_o[h*d + e][n],
+ * i.e. head h contributes O[b][h][t][:] times its own (d x d_y) block of W_o.
+ *   O    float  [B][H][T][d]    the attention output (Eq. 12)
+ *   Wot  float  [d_y][H*d]      W_o stored transposed: Wot[n][h*d + e] = W_o[h*d + e][n]
+ *   Y    double [B][T][d_y]     rows at positions >= len_b are zero
+ */
+void psattn_oracle_project_out(const float *O, const float *Wot, int B, int H, int T, int d, int dy,
+                               const int *lengths, double *Y, int nthreads) {
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(nthreads > 0 ? nthreads : 1) schedule(static)
+#endif
+    for (long bt = 0; bt < (long)B * T; ++bt) {
+        int b = (int)(bt / T), t = (int)(bt % T);
+        int L = seq_len(lengths, b, T);
+        for (int n = 0; n < dy; ++n) {
+            double acc = 0.0;
+            if (t < L)
+                for (int h = 0; h < H; ++h) {
+                    const float *o = O + (((size_t)b * H + h) * T + t) * d;
+                    const float *w = Wot + (size_t)n * H * d + (size_t)h * d;
+                    for (int e = 0; e < d; ++e) acc += (double)o[e] * (double)w[e];
+                }
+            Y[(size_t)bt * dy + n] = acc;
+        }
     }
 }
 

@@ -218,3 +218,19 @@ def project_qkv(X, Wt, H, lengths=None, nthreads=1):
     lib.psattn_oracle_project_qkv(xp, wp, B, T, dx, int(H), d, lp, out.ctypes.data_as(_f64p),
                                   int(nthreads))
     return out[0], out[1], out[2]
+
+
+def project_out(O, Wot, lengths=None, nthreads=1):
+    """The output matrix of the attention module: Y[b, t, :] = sum_h O[b, h, t, :] W_o^h.  O [B, H, T, d];
+    Wot [d_y, H*d] holds W_o transposed (Wot[n, h*d + e] = W_o[h*d + e, n]).  Returns float64 [B, T, d_y],
+    zero at padded positions."""
+    lib = _load()
+    O, op = _f32(O)
+    Wot, wp = _f32(Wot)
+    B, H, T, d = O.shape
+    assert Wot.ndim == 2 and Wot.shape[1] == H * d
+    dy = int(Wot.shape[0])
+    lengths, lp = _i32(lengths)
+    Y = np.zeros((B, T, dy), dtype=np.float64)
+    lib.psattn_oracle_project_out(op, wp, B, H, T, d, dy, lp, Y.ctypes.data_as(_f64p), int(nthreads))
+    return Y

@@ -530,3 +530,61 @@ def test_projection_workload_generator():
     np.testing.assert_array_equal(a["Wt"], b["Wt"])
     Q, _, _ = orc.project_qkv(a["X"], a["Wt"], w.H)
     assert 0.8 < Q.std() < 1.2                                           # unit-variance activations by construction
+
+
+# ---- the output matrix that merges the heads (Sec. 2.2 Eq. 5, Sec. 3.1) ---------------------------
+
+def test_output_projection_equals_library_matmul_of_concatenated_heads():
+    rng = np.random.default_rng(31)
+    B, H, T, d, dy = 2, 3, 7, 4, 5
+    O = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    Wot = rng.standard_normal((dy, H * d)).astype(np.float32)
+    lengths = np.array([7, 4], dtype=np.int32)
+    Y = orc.project_out(O, Wot, lengths)
+    concat = O.transpose(0, 2, 1, 3).reshape(B, T, H * d).astype(np.float64)     # heads side by side
+    want = concat @ Wot.astype(np.float64).T
+    want[1, 4:] = 0.0
+    np.testing.assert_allclose(Y, want, rtol=0, atol=1e-12)
+
+
+def test_output_projection_one_hot_identity_and_linearity():
+    rng = np.random.default_rng(32)
+    B, H, T, d = 1, 3, 5, 4
+    O = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    # identity: the output is the concatenation of the heads (head h lands in columns h*d .. h*d+d-1)
+    Y = orc.project_out(O, np.eye(H * d, dtype=np.float32))
+    for h in range(H):
+        np.testing.assert_array_equal(Y[0, :, h * d:(h + 1) * d], O[0, h].astype(np.float64))
+    # one weight only, Wot[n0, k0] = 1: column n0 of Y reads feature k0 = (h0, e0); a transposed or
+    # head-swapped operand reads another one
+    dy, n0, h0, e0 = 6, 4, 2, 1
+    Wot = np.zeros((dy, H * d), dtype=np.float32)
+    Wot[n0, h0 * d + e0] = 1.0
+    Y = orc.project_out(O, Wot)
+    np.testing.assert_array_equal(Y[0, :, n0], O[0, h0, :, e0].astype(np.float64))
+    assert np.count_nonzero(np.delete(Y, n0, axis=2)) == 0
+    # linear in O and in the weights
+    W1 = rng.standard_normal((dy, H * d)).astype(np.float32)
+    O2 = rng.standard_normal((B, H, T, d)).astype(np.float32)
+    np.testing.assert_allclose(orc.project_out(O + O2, W1), orc.project_out(O, W1) + orc.project_out(O2, W1),
+                               atol=1e-5)
+
+
+def test_output_projection_of_unselected_rows_is_one_row():
+    """Eq. 12 with the mean(V) fill: every non-selected row of a unit is the same vector, so their rows of Y
+    are identical (what the library's shortcut relies on); the selected rows differ."""
+    B, H, T, d, c = 1, 2, 30, 8, 1.0
+    Q, K, V, idx, lengths = _rand(B, H, T, d, 33, brute.n_count(c, T))
+    O, sel, _ = orc.forward(Q, K, V, idx, lengths, c=c)
+    rng = np.random.default_rng(34)
+    Wot = rng.standard_normal((6, H * d)).astype(np.float32)
+    Y = orc.project_out(O.astype(np.float32), Wot)
+    chosen = set(int(x) for x in sel.reshape(-1) if x >= 0)
+    rest = [t for t in range(T) if t not in chosen]
+    assert len(rest) > 2 and len(chosen) > 0
+    for t in rest[1:]:
+        np.testing.assert_array_equal(Y[0, t], Y[0, rest[0]])
+    vbar = orc.mean_v(V, lengths).astype(np.float32).astype(np.float64)
+    want = sum(vbar[0, h] @ Wot[:, h * d:(h + 1) * d].astype(np.float64).T for h in range(H))
+    np.testing.assert_allclose(Y[0, rest[0]], want, atol=1e-5)
+    assert any(not np.allclose(Y[0, t], Y[0, rest[0]]) for t in chosen)

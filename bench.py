@@ -620,6 +620,23 @@ def run_variants(cx, w, r, dense_ms):
                 "frac_of_tensor_peak": p_flops / (p_ms * 1e-3) / 1e12 / tf_peak[0],
                 "peak_kind": "of " + tf_peak[1], "d_x": dx, "device_status": plan.psattn_read_status()}
         del pO, pX
+        # the output matrix behind the path (Sec. 2.2 Eq. 5): the broadcast-plus-corrections form that uses the
+        # structure of O (one fill row per unit plus u selected rows) beside the dense tcgen05 product
+        for s in range(n_sets):
+            r["step"](s)                                     # O and sel of every buffer set belong together
+        rng = np.random.default_rng(w.seed + 31)
+        Wo = torch.from_numpy((rng.standard_normal((dx, dx)) / np.sqrt(dx)).astype(np.float32)).to("cuda", tdt)
+        Ys = [torch.empty((w.B, w.T, dx), dtype=tdt, device="cuda") for _ in range(n_sets)]
+        o_flops = 2.0 * dx * dx * sum(int(L) for L in host0["lengths"])
+        for key, use_sel in (("output_projection_shortcut", True), ("output_projection_dense", False)):
+            def out_proj(s, use_sel=use_sel):
+                d = sets[s]
+                plan.psattn_project_out(d["O"], d["sel"] if use_sel else None, d["lengths"], Wo, Ys[s])
+            o_ms = timed(out_proj, nk)
+            variants[key] = {"ms_per_step": o_ms, "d_y": dx, "dense_equivalent_tflops": o_flops / (o_ms * 1e-3) / 1e12,
+                             "written_gbs": w.B * w.T * dx * elem / (o_ms * 1e-3) / 1e9,
+                             "device_status": plan.psattn_read_status()}
+        del Ys
     return variants
 
 

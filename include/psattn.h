@@ -167,6 +167,23 @@ int psattn_project_qkv(psattn_plan_t *plan, const void *X, const void *Wt, int32
                        const int32_t *lengths, void *Q, void *K, void *V, float *vbar,
                        void *workspace, size_t workspace_bytes, void *stream);
 
+/* The output matrix of the attention module, which merges the heads (Sec. 2.2, Eq. 5: the module inside the
+ * Conformer block; Sec. 3.1: its heads):  Y[b][t][n] = sum_h sum_e O[b][h][t][e] W_o^h[e][n].  All pointers device.
+ *   O        the attention output, plan type, descriptor's o strides (what psattn_forward wrote)
+ *   sel_idx  the index sets that psattn_forward wrote for this O ([B][H][u_max], ascending, -1 padded), or NULL
+ *   Wot      [d_y][H * 64] dense, plan type: W_o transposed, Wot[n][h * 64 + e] = W_o^h[e][n]
+ *   Y        [B][T_max][d_y] dense, plan type; rows at positions >= lengths[b] are NOT written
+ * With sel_idx, the mean(V) fill and bf16 (u_max <= 64, H <= 32, d_y a multiple of 8) the call uses the structure
+ * Eq. 12 gives O - every valid row of a unit that its index set does not list equals one fill row F_h - and
+ * computes Y[b][t][:] = sum_h F_h W_o^h for all positions plus (O[b][h][t][:] - F_h) W_o^h for the listed ones:
+ * O(B H u 64 d_y) products instead of O(B T H 64 d_y).  F_h is read from O at the first valid position the set
+ * leaves out, so O must really have that structure (rows changed after psattn_forward are not seen).
+ * With sel_idx == NULL (any O), the own-value fill, or shapes outside those limits: one dense product (tcgen05 for
+ * bf16 with d_y a multiple of 64; one thread per output element for fp32, other d_y, or PSATTN_PATH_STAGED). */
+int psattn_project_out(psattn_plan_t *plan, const void *O, const int32_t *sel_idx, const int32_t *lengths,
+                       const void *Wot, int32_t d_y, void *Y, void *workspace, size_t workspace_bytes,
+                       void *stream);
+
 /* Step (c) only (Sec. 3.2): top-u positions of M (fp32 [B][H][T_max]) among i < lengths[b]. */
 int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
                   int32_t *sel_idx, void *workspace, size_t workspace_bytes, void *stream);

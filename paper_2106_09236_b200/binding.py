@@ -22,7 +22,7 @@ EXPORTS = [
     "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_exact_measure", "psattn_select",
     "psattn_mean_v", "psattn_attend_rows", "psattn_dense_forward", "psattn_read_status",
     "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc", "psattn_project_qkv",
-    "psattn_probe_gather",
+    "psattn_probe_gather", "psattn_project_out",
 ]
 
 
@@ -79,6 +79,7 @@ def load(build_if_missing: bool = True):
     lib.psattn_select.argtypes = [vp] * 5 + [sz, vp]
     lib.psattn_project_qkv.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.psattn_mean_v.argtypes = [vp] * 5 + [sz, vp]
+    lib.psattn_project_out.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     lib.psattn_attend_rows.argtypes = [vp] * 6 + [i32, vp, vp, sz, vp]
     lib.psattn_dense_forward.argtypes = [vp] * 7 + [sz, vp]
     lib.psattn_read_status.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -240,6 +241,18 @@ class Plan:
                                            _ptr(outs[0]), _ptr(outs[1]), _ptr(outs[2]), _ptr(vbar), ws, n,
                                            _stream()), self.handle)
         return tuple(outs)
+
+    def psattn_project_out(self, O, sel_idx, lengths, Wot, Y=None):
+        """Y[b, t, :] = sum_h O[b, h, t, :] W_o^h; Wot [d_y, H*64] holds W_o transposed.  With sel_idx (the index
+        sets psattn_forward wrote for this O) the broadcast-plus-corrections form runs, with None the dense product.
+        Rows at padded positions of a freshly allocated Y are zero (the kernels do not write them)."""
+        d_y = int(Wot.shape[0])
+        if Y is None:
+            Y = torch.zeros((self.B, self.T_max, d_y), dtype=self.dtype, device=O.device)
+        ws, n = self._ws()
+        _check(self.lib.psattn_project_out(self.handle, _ptr(O), _ptr(sel_idx), _ptr(lengths), _ptr(Wot), d_y,
+                                           _ptr(Y), ws, n, _stream()), self.handle)
+        return Y
 
     def psattn_select(self, M, lengths, sel_idx=None):
         if sel_idx is None:

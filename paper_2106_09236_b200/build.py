@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpsattn.so")
-SOURCES = ["psattn_api.cu", "psattn_staged.cu", "psattn_noalloc.cu", "psattn_attend_tc.cu", "psattn_measure_mma.cu", "psattn_measure_shared.cu", "psattn_exact_measure.cu", "psattn_project.cu", "psattn_attend64.cu", "psattn_fused.cu", "psattn_probe.cu"]
+SOURCES = ["psattn_api.cu", "psattn_staged.cu", "psattn_noalloc.cu", "psattn_attend_tc.cu", "psattn_measure_mma.cu", "psattn_measure_shared.cu", "psattn_exact_measure.cu", "psattn_project.cu", "psattn_attend64.cu", "psattn_fused.cu", "psattn_probe.cu", "psattn_project_out.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC",

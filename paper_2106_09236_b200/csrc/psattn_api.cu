@@ -484,6 +484,24 @@ extern "C" int psattn_project_qkv(psattn_plan_t *plan, const void *X, const void
     return PSATTN_OK;
 }
 
+extern "C" int psattn_project_out(psattn_plan_t *plan, const void *O, const int32_t *sel_idx, const int32_t *lengths,
+                                  const void *Wot, int32_t d_y, void *Y, void *workspace, size_t workspace_bytes,
+                                  void *stream) {
+    if (!plan || !O || !Wot || !Y) return PSATTN_ERR_NULL;
+    if (d_y < 1 || d_y > (1 << 20)) return PSATTN_ERR_BAD_DESC;
+    if (!aligned16(O) || !aligned16(Wot) || !aligned16(Y)) return PSATTN_ERR_MISALIGNED;
+    int rc = check_ws(plan, workspace, workspace_bytes);
+    if (rc) return rc;
+    const psattn_desc_t &d = plan->desc;
+    Geom g = make_geom(plan, lengths, workspace);
+    // the shortcut needs Eq. 12's structure with the mean(V) fill; any other O goes through the dense product
+    const int mode = d.path == PSATTN_PATH_STAGED ? 2 : (sel_idx != nullptr && d.fill_mode == PSATTN_FILL_MEAN_V ? 0 : 1);
+    cudaError_t e = launch_project_out(d.dtype, mode, g, d_y, O, sel_idx, Wot, Y, static_cast<cudaStream_t>(stream));
+    if (e == cudaErrorNotSupported) return PSATTN_ERR_UNSUPPORTED;
+    PSATTN_CU(e);
+    return PSATTN_OK;
+}
+
 extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
                              int32_t *sel_idx, void *workspace, size_t workspace_bytes,
                              void *stream) {

@@ -112,6 +112,12 @@ cudaError_t merge_attend_splits(int out_is_bf16, const Geom &g, const int *rows,
 size_t project_vpart_floats(int B, int H, int T);
 cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx, const void *X, const void *Wt, void *Q,
                                void *K, void *V, float *vbar, float *vpart, cudaStream_t st);
+// The output matrix of the attention module: Y [B][T][dy] = sum_h O[b][h][t][:] W_o^h, Wot [dy][H * 64].
+// mode 0: with an index set `sel` ([B][H][g.u_max], as psattn_forward writes it) and the mean(V) fill, the
+// broadcast-plus-corrections form; otherwise (and with mode 1) the dense tcgen05 GEMM; mode 2 or fp32: one
+// thread per output element.  Rows at padded positions are not written.
+cudaError_t launch_project_out(int dtype, int mode, const Geom &g, int dy, const void *O, const int *sel, const void *Wot,
+                               void *Y, cudaStream_t st);
 cudaError_t launch_fill(int dtype, const Geom &g, const void *V, const int *sel, const float *vbar,
                         void *O, int own_v, cudaStream_t st);
 

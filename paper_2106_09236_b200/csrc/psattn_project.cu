@@ -39,7 +39,10 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *m, uin
 }
 
 struct ProjArgs {
-    int B, H, T, dx;
+    int B, H, T, dx;                              // H: 64-column blocks per role (the heads of the outputs)
+    int n_blocks;                                 // 64-column blocks of all roles together (3 H for Q, K, V)
+    int x_heads;                                  // 0: X is [B][T][dx] (3-D tensor map); 1: X is in the attention layout
+    int pos_t, pos_h, pos_b;                      //    [B][H_in][T][64] (4-D map, these coordinate slots), dx = H_in * 64
     int tiles_per_seq, n_tiles_n, n_tiles;        // 128-token tiles per sequence, 192-column tiles, all tiles
     long long qs[3], ks[3], vs[3];                // element strides (b, h, t) of the three outputs
     __nv_bfloat16 *Q, *K, *V;
@@ -104,7 +107,13 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
                     if (!mbar_wait(&empty[s], ph ^ 1u)) { atomicOr(a.status, kStatusWaitExpired); *abort_flag = 1; break; }
                     uint8_t *sa = smem + s * kPjStage;
                     mbar_expect_tx(&full[s], kPjStage);
-                    tma_load_3d(sa, &tmX, &full[s], kb * kPjK, tt * kPjM, b);
+                    if (a.x_heads) {                           // slab kb = head kb of the attention layout
+                        const int t0 = tt * kPjM;
+                        tma_load_4d(sa, &tmX, &full[s], 0, a.pos_t == 1 ? t0 : (a.pos_h == 1 ? kb : b),
+                                    a.pos_t == 2 ? t0 : (a.pos_h == 2 ? kb : b), a.pos_t == 3 ? t0 : (a.pos_h == 3 ? kb : b));
+                    } else {
+                        tma_load_3d(sa, &tmX, &full[s], kb * kPjK, tt * kPjM, b);
+                    }
                     tma_load_2d(sa + kPjBytesA, &tmW, &full[s], kb * kPjK, n * kPjN);
                 }
             }
@@ -165,7 +174,7 @@ __global__ void __launch_bounds__(kPjThreads, 1) k_project_qkv(ProjArgs a, const
                 break;
             }
             tc_fence_after();
-            const int n_cc = min(kPjN / 64, 3 * a.H - n * (kPjN / 64));   // 64-column blocks of this tile
+            const int n_cc = min(kPjN / 64, a.n_blocks - n * (kPjN / 64));   // 64-column blocks of this tile
             const uint32_t tacc = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kPjAccCols;
             uint32_t ra[64], rb[64];                           // two blocks in flight: the next one loads while
             tmem_ld32_issue(tacc, ra);                         // the current one is converted and stored
@@ -324,6 +333,7 @@ cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx,
     if (g.B * g.H == 0) return cudaSuccess;
     ProjArgs a;
     a.B = g.B; a.H = g.H; a.T = g.T; a.dx = dx;
+    a.n_blocks = 3 * g.H; a.x_heads = 0; a.pos_t = a.pos_h = a.pos_b = 0;
     a.tiles_per_seq = (g.T + kPjM - 1) / kPjM;
     a.n_tiles_n = (3 * g.H * 64 + kPjN - 1) / kPjN;
     a.n_tiles = g.B * a.tiles_per_seq * a.n_tiles_n;
@@ -385,6 +395,50 @@ cudaError_t launch_project_qkv(int dtype, int force_simt, const Geom &g, int dx,
         if (vbar) { k_project_vbar_simt<float><<<g.B * g.H, 64, 0, st>>>(a, (const float *)V, vbar); note_launch(); }
     }
     return cudaGetLastError();
+}
+
+
+bool make_rows_map(CUtensorMap *map, const void *base, const Geom &g, const long long s[3], int box_rows,
+                   int swizzle128, int pos[3]);
+
+// Dense form of the output matrix of the attention module (see psattn_project_out.cu): Y[b][t][:] =
+// sum_h O[b][h][t][:] W_o^h as ONE GEMM on the kernel above, the K dimension running over the heads of the
+// attention layout (slab kb = head kb, fetched through a 4-D tensor map of O), the 64-column blocks of Y
+// standing where the heads of one role stand for the projections.  bf16, dy a multiple of 64.
+// cudaErrorNotSupported: no tensor map for the layout.
+cudaError_t launch_project_out_dense(const Geom &g, int dy, const void *O, const void *Wot, void *Y, cudaStream_t st) {
+    if (g.B * g.H == 0) return cudaSuccess;
+    EncodeTiledFnP enc = proj_encode_fn();
+    if (!enc || dy % 64 != 0 || dy < 64) return cudaErrorNotSupported;
+    ProjArgs a;
+    a.B = g.B; a.H = dy / 64; a.T = g.T; a.dx = g.H * 64;
+    a.n_blocks = dy / 64; a.x_heads = 1;
+    a.tiles_per_seq = (g.T + kPjM - 1) / kPjM;
+    a.n_tiles_n = (dy + kPjN - 1) / kPjN;
+    a.n_tiles = g.B * a.tiles_per_seq * a.n_tiles_n;
+    // Y [B][T][dy] seen as [B][dy / 64][T][64]: block stride 64, token stride dy
+    const long long ys[3] = {(long long)g.T * dy, 64, dy};
+    for (int k = 0; k < 3; ++k) { a.qs[k] = ys[k]; a.ks[k] = ys[k]; a.vs[k] = ys[k]; }
+    a.Q = (__nv_bfloat16 *)Y; a.K = nullptr; a.V = nullptr;
+    a.lengths = g.lengths; a.status = g.status; a.vpart = nullptr;
+    CUtensorMap tmX, tmW;
+    int pos[3];
+    if (!make_rows_map(&tmX, O, g, g.os, kPjM, 1, pos)) return cudaErrorNotSupported;
+    a.pos_t = pos[0]; a.pos_h = pos[1]; a.pos_b = pos[2];
+    const cuuint64_t wdim[2] = {(cuuint64_t)a.dx, (cuuint64_t)dy};
+    const cuuint64_t wstr[1] = {(cuuint64_t)a.dx * 2};
+    const cuuint32_t wbox[2] = {kPjK, kPjN}, one2[2] = {1, 1};
+    if (enc(&tmW, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(Wot), wdim, wstr, wbox, one2,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorNotSupported;
+    static SmemGrant grant;
+    if (cudaError_t e = grant_dynamic_smem(k_project_qkv, grant, kPjSmem)) return e;
+    const int sms = device_sm_count();
+    cudaError_t e = launch_pdl(k_project_qkv, dim3((unsigned)(a.n_tiles < sms ? a.n_tiles : sms)), dim3(kPjThreads), kPjSmem,
+                               st, a, tmX, tmW);
+    note_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace psattn

@@ -312,10 +312,10 @@ static int run_attend(psattn_plan_t *plan, const Geom &g, const void *Q, const v
         if (e != cudaErrorNotSupported || vbar != nullptr) return cuda_fail(plan, e);
     }
     if (d.dtype == PSATTN_BF16 && d.path != PSATTN_PATH_STAGED) {
-        // key splits: enough CTAs to cover the SMs about twice, never more splits than 128-key tiles
+        // key splits: enough CTAs (256 rows each, one per SM) to cover the SMs, never more splits than 128-key tiles
         const int tiles = (d.T_max + 127) / 128;
-        const long long ctas = (long long)d.B * d.H * ((n_rows + 127) / 128);
-        int splits = (int)((2 * device_sm_count() + ctas - 1) / (ctas > 0 ? ctas : 1));
+        const long long ctas = (long long)d.B * d.H * ((n_rows + 255) / 256);
+        int splits = (int)((device_sm_count() + ctas - 1) / (ctas > 0 ? ctas : 1));
         if (splits > plan->n_splits) splits = plan->n_splits;
         if (splits > tiles) splits = tiles;
         if (splits < 1 || rows == nullptr) splits = 1;
@@ -552,13 +552,8 @@ extern "C" int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const vo
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const psattn_desc_t &d = plan->desc;
     Geom g = make_geom(plan, lengths, workspace);
-    // zero rows at padded positions: a fill with an empty selection and a zero "mean" would
-    // also overwrite valid rows, so fill first (mean value irrelevant) and let attention
-    // overwrite every valid row.
-    int *sel = ws_at<int>(workspace, plan->off_sel);
-    PSATTN_CU(cudaMemsetAsync(sel, 0xff, (size_t)d.B * d.H * plan->u_max * sizeof(int), st));
-    PSATTN_CU(cudaMemsetAsync(ws_at<float>(workspace, plan->off_vbar), 0, (size_t)d.B * d.H * kD * sizeof(float), st));
-    PSATTN_CU(launch_fill(d.dtype, g, V, sel, ws_at<float>(workspace, plan->off_vbar), O, 0, st));
+    // every position is a listed row (identity list): the attention kernels write the valid rows and the zero
+    // rows at padded positions themselves
     return run_attend(plan, g, Q, K, V, nullptr, d.T_max, 0, O, 0, 0, 1, 0, workspace, st);
 }
 

@@ -246,7 +246,8 @@ __global__ void __launch_bounds__(128) k_attend(Geom g, const DT *__restrict__ Q
     const bool row_ok = i >= 0 && i < L;
     // where the finished row goes: at its position i of O, or at its slot r of a row-list output
     OT *dst = nullptr;
-    if (out_by_position) { if (row_ok) dst = out + unit_off(g.os, b, h) + (long long)i * g.os[2]; }
+    // (with the identity list every position is a row: the padded ones get their zero rows here)
+    if (out_by_position) { if (row_ok || (rows == nullptr && i < g.T)) dst = out + unit_off(g.os, b, h) + (long long)i * g.os[2]; }
     else dst = out + (long long)unit * out_unit_stride + (long long)r * out_row_stride;
 
     float m = -INFINITY, l = 0.f;
@@ -343,7 +344,7 @@ __global__ void __launch_bounds__(256) k_attend_combine(Geom g, const int *__res
     const bool row_ok = i >= 0 && i < L;
     OT *dst;
     if (out_by_position) {
-        if (!row_ok) return;
+        if (!row_ok && !(rows == nullptr && i < g.T)) return;   // identity list: padded positions get zero rows
         dst = out + unit_off(g.os, b, h) + (long long)i * g.os[2];
     } else {
         dst = out + (long long)unit * out_unit_stride + (long long)r * out_row_stride;

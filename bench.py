@@ -681,6 +681,38 @@ def run_dense(cx, w, r):
             "score_matrix_bytes_if_materialised": 4 * w.B * w.H * w.T * w.T}
 
 
+def run_phases(cx, w):
+    """Per-phase times of the fused forward kernel (one CTA per unit, phases in series): a build of the library
+    with -DPSATTN_PHASE_STAMPS accumulates, per CTA, the time between block-wide barriers at the phase ends."""
+    torch, ps = cx.torch, cx.ps
+    tdt, elem = torch.bfloat16, 2
+    n_cols = max(ps.psattn_count(w.c, L) for L in range(1, w.T + 1))
+    plan = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols, path=ps.PSATTN_PATH_FUSED)
+    sets, _, _ = make_sets(cx, w, n_cols, plan, tdt, elem)
+
+    def step(s):
+        d = sets[s]
+        plan.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], d["sel"])
+    for k in range(5):
+        step(k % len(sets))
+    torch.cuda.synchronize()
+    acc = plan.workspace[64:128].view(torch.int64)
+    acc.zero_()
+    steps = 200
+    ms = cx.time_once(lambda k: step(k % len(sets)), steps)
+    torch.cuda.synchronize()
+    a = acc.cpu().numpy()
+    ctas = max(int(a[0]), 1)
+    names = ["wait for the unit's keys (TMA, cold)", "steps (a)+(b): sampled scores, measure", "step (c): top-u select",
+             "step (d): attention of the selected rows (+ column sums of V)", "step (e): fill"]
+    phases = {names[k]: float(a[k + 1]) / ctas / 1e3 for k in range(5)}
+    out = {"phases": "k_forward_fused, mean over %d CTA runs (%d steps, direct calls)" % (ctas, steps), "workload": w.name,
+           "us_per_cta": phases, "us_sum": sum(phases.values()), "us_per_step_this_run": ms * 1e3,
+           "note": "stamps cost a few hundred ns per CTA; the step time of the regular build is the one bench.py reports"}
+    plan.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -690,6 +722,8 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=sorted(wl.WORKLOADS))
     ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--probe", default=None, choices=["gather"], help="run only the named microbenchmark")
+    ap.add_argument("--phases", action="store_true",
+                    help="per-phase times of the fused forward kernel (builds a stamped copy of the library first)")
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of CUDA-graph replays")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense comparator timing")
@@ -701,6 +735,14 @@ def main():
         run_reference(args, w)
         return
 
+    if args.phases:
+        from paper_2106_09236_b200 import build as lib_build
+        os.environ["PSATTN_LIBRARY"] = lib_build.build(phase_stamps=True)
+        cx = Ctx(args)
+        wp = w if w.name != HEADLINE else wl.WORKLOADS[OTHER]          # the fused kernel takes T_max <= ~1100
+        if cx.rank == 0:
+            print(json.dumps(run_phases(cx, wp)), flush=True)
+        return
     cx = Ctx(args)
     probe = gather_probe(cx)
     if args.probe == "gather":

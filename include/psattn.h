@@ -118,6 +118,15 @@ int psattn_count(double c, int len);
  * the host and uploads them, and records the current device.  *out is NULL on failure. */
 int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out);
 int psattn_plan_destroy(psattn_plan_t *plan);
+/* Test hook for the bounded device-side waits.  Every wait of a kernel on a barrier (a TMA copy, a tensor-core
+ * product) gives up after a limit (1 s), sets PSATTN_STATUS_WAIT_EXPIRED and lets the kernel unwind and return.
+ * This call shortens the limit (wait_limit_ns, 0 = the default of 1 s, at most 10 s) for the kernels that take it
+ * from the plan (the fused forward kernel and the long-row-list / dense attention kernel) and, with
+ * extra_expected_bytes > 0, makes the first TMA barrier of those kernels expect that many bytes more than are ever
+ * sent, so that the wait really runs out - without any invalid access.  Results of such a call are invalid by
+ * design; pass (0, 0) to return to normal operation. */
+int psattn_plan_debug_waits(psattn_plan_t *plan, uint64_t wait_limit_ns, uint32_t extra_expected_bytes);
+
 /* Largest u and U over len in [0, T_max]: the widths of sel_idx and the minimum idx_cols. */
 int psattn_plan_limits(const psattn_plan_t *plan, int32_t *u_max, int32_t *U_max);
 /* Bytes of device workspace every call below needs (the same size for all of them). */

@@ -22,7 +22,7 @@ EXPORTS = [
     "psattn_forward", "psattn_forward_with_selection", "psattn_measure", "psattn_exact_measure", "psattn_select",
     "psattn_mean_v", "psattn_attend_rows", "psattn_dense_forward", "psattn_read_status",
     "psattn_plan_enable_host_io", "psattn_forward_host", "psattn_mean_v_noalloc", "psattn_project_qkv",
-    "psattn_probe_gather", "psattn_project_out",
+    "psattn_probe_gather", "psattn_project_out", "psattn_plan_debug_waits",
 ]
 
 
@@ -56,7 +56,10 @@ def load(build_if_missing: bool = True):
     if _lib is not None:
         return _lib
     path = _build.LIB
-    if build_if_missing:
+    override = os.environ.get("PSATTN_LIBRARY")          # another build of the same library (the benchmark's --phases mode)
+    if override:
+        path = override
+    elif build_if_missing:
         path = _build.build()
     if not os.path.exists(path):
         raise PsattnError("libpsattn.so is missing: run paper_2106_09236_b200/build.py")
@@ -86,6 +89,7 @@ def load(build_if_missing: bool = True):
     lib.psattn_plan_enable_host_io.argtypes = [vp]
     lib.psattn_forward_host.argtypes = [vp] * 9
     lib.psattn_mean_v_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.psattn_plan_debug_waits.argtypes = [vp, ctypes.c_uint64, ctypes.c_uint32]
     lib.psattn_probe_gather.argtypes = [i32, vp, ctypes.c_int64, i32, i32, i32, vp, vp]
     _lib = lib
     return lib
@@ -293,6 +297,10 @@ class Plan:
         _check(self.lib.psattn_read_status(self.handle, _ptr(self.workspace), _stream(),
                                            ctypes.byref(bits)), self.handle)
         return bits.value
+
+    def psattn_plan_debug_waits(self, wait_limit_ns=0, extra_expected_bytes=0):
+        """Test hook: shorten the bounded device-side waits and/or make the first TMA barrier never complete."""
+        _check(self.lib.psattn_plan_debug_waits(self.handle, int(wait_limit_ns), int(extra_expected_bytes)), self.handle)
 
     def psattn_plan_enable_host_io(self):
         _check(self.lib.psattn_plan_enable_host_io(self.handle), self.handle)

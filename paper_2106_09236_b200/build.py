@@ -26,12 +26,16 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h"))]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "psattn.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, phase_stamps: bool = False) -> str:
+    """Builds the library.  phase_stamps: a second library, libpsattn_stamps.so, whose fused forward kernel
+    accumulates per-phase times (-DPSATTN_PHASE_STAMPS); only the benchmark's --phases mode uses it."""
+    if phase_stamps:
+        return _build_variant("libpsattn_stamps.so", ["-DPSATTN_PHASE_STAMPS"], ".stamps.o")
     if not force and not needs_build():
         return LIB
     objs = []
@@ -48,6 +52,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart"])
     os.replace(tmp, LIB)
     return LIB
+
+
+def _build_variant(name: str, extra: list, suffix: str) -> str:
+    out = os.path.join(HERE, name)
+    objs = []
+    for src in SOURCES:
+        obj = os.path.join(CSRC, src.replace(".cu", suffix))
+        subprocess.check_call([_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj])
+        objs.append(obj)
+    tmp = out + ".tmp.%d" % os.getpid()
+    subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart"])
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":

@@ -32,6 +32,8 @@ struct psattn_plan {
     // side stream of the staged schedule: the fill of step (e) runs there while steps (a)-(c) run on the caller's
     cudaStream_t side_stream;
     cudaEvent_t side_ev[2];       // [0]: fork (recorded on the caller's stream), [1]: join (recorded on the side stream)
+    unsigned long long wait_ns;   // limit of the bounded device-side waits (psattn_plan_debug_waits)
+    unsigned debug_extra_tx;
 };
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -143,6 +145,8 @@ extern "C" int psattn_plan_create(const psattn_desc_t *desc, psattn_plan_t **out
     p->device = dev;
     p->u_max = u_max;
     p->U_max = U_max;
+    p->wait_ns = 1000ull * 1000ull * 1000ull;
+    p->debug_extra_tx = 0u;
     p->n_chunks = (d.T_max + kColsumRows - 1) / kColsumRows;
     p->n_splits = (d.T_max + kSplitKeys - 1) / kSplitKeys;       // what the partial buffers are sized for
     {
@@ -196,6 +200,14 @@ extern "C" int psattn_plan_destroy(psattn_plan_t *p) {
     return PSATTN_OK;
 }
 
+extern "C" int psattn_plan_debug_waits(psattn_plan_t *p, uint64_t wait_limit_ns, uint32_t extra_expected_bytes) {
+    if (!p) return PSATTN_ERR_NULL;
+    if (wait_limit_ns > 10ull * 1000ull * 1000ull * 1000ull) return PSATTN_ERR_BAD_DESC;
+    p->wait_ns = wait_limit_ns ? wait_limit_ns : 1000ull * 1000ull * 1000ull;
+    p->debug_extra_tx = extra_expected_bytes;
+    return PSATTN_OK;
+}
+
 extern "C" int psattn_plan_limits(const psattn_plan_t *p, int32_t *u_max, int32_t *U_max) {
     if (!p) return PSATTN_ERR_NULL;
     if (u_max) *u_max = p->u_max;
@@ -244,6 +256,8 @@ static Geom make_geom(const psattn_plan_t *p, const int32_t *lengths, void *ws) 
     g.u_tab = p->d_tables;
     g.U_tab = p->d_tables + d.T_max + 1;
     g.status = reinterpret_cast<unsigned *>(static_cast<char *>(ws) + p->off_status);
+    g.wait_ns = p->wait_ns;
+    g.debug_extra_tx = p->debug_extra_tx;
     return g;
 }
 

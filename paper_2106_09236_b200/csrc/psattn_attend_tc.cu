@@ -181,10 +181,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
                 const int c1 = a.pos_t == 1 ? key0 : (a.pos_h == 1 ? h : b);
                 const int c2 = a.pos_t == 2 ? key0 : (a.pos_h == 2 ? h : b);
                 const int c3 = a.pos_t == 3 ? key0 : (a.pos_h == 3 ? h : b);
-                if (!mbar_wait(&k_empty[s], ph ^ 1u)) { give_up(); break; }
-                mbar_expect_tx(&k_full[s], kTileBytes);
+                if (!mbar_wait(&k_empty[s], ph ^ 1u, g.wait_ns)) { give_up(); break; }
+                mbar_expect_tx(&k_full[s], kTileBytes + (t == 0 ? g.debug_extra_tx : 0u));
                 tma_load_4d(smem + kOffK + s * kTileBytes, &tmK, &k_full[s], 0, c1, c2, c3);
-                if (!mbar_wait(&v_empty[s], ph ^ 1u)) { give_up(); break; }
+                if (!mbar_wait(&v_empty[s], ph ^ 1u, g.wait_ns)) { give_up(); break; }
                 mbar_expect_tx(&v_full[s], kTileBytes);
                 tma_load_4d(smem + kOffV + s * kTileBytes, &tmV, &v_full[s], 0, c1, c2, c3);
             }
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
                 umma_commit(&s_full[w]);
             };
             bool alive = !*abort_flag;
-            if (alive && !mbar_wait(&k_full[0], 0u)) { give_up(); alive = false; }
+            if (alive && !mbar_wait(&k_full[0], 0u, g.wait_ns)) { give_up(); alive = false; }
             if (alive) {
                 tc_fence_after();
                 for (int w = 0; w < n_wg; ++w) issue_s(w, 0);
@@ -219,8 +219,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
                 const int s = t % kTcStages, sn = (t + 1) % kTcStages;
                 const uint32_t ph = (uint32_t)((t / kTcStages) & 1), phn = (uint32_t)(((t + 1) / kTcStages) & 1);
                 for (int w = 0; w < n_wg; ++w) {
-                    if (!mbar_wait(&p_ready[w], (uint32_t)(t & 1))) { give_up(); alive = false; break; }
-                    if (w == 0 && !mbar_wait(&v_full[s], ph)) { give_up(); alive = false; break; }
+                    if (!mbar_wait(&p_ready[w], (uint32_t)(t & 1), g.wait_ns)) { give_up(); alive = false; break; }
+                    if (w == 0 && !mbar_wait(&v_full[s], ph, g.wait_ns)) { give_up(); alive = false; break; }
                     tc_fence_after();
                     const uint64_t pa = dp + (uint64_t)(2 * w) * kTile16, va = dv + (uint64_t)s * kTile16;
 #pragma unroll
@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
                                   kIdescO, (t > 0 || k > 0) ? 1u : 0u);
                     if (w == n_wg - 1) umma_commit(&v_empty[s]);
                     if (t + 1 < n_tiles) {
-                        if (w == 0 && !mbar_wait(&k_full[sn], phn)) { give_up(); alive = false; break; }
+                        if (w == 0 && !mbar_wait(&k_full[sn], phn, g.wait_ns)) { give_up(); alive = false; break; }
                         tc_fence_after();
                         issue_s(w, t + 1);
                         if (w == n_wg - 1) umma_commit(&k_empty[sn]);
@@ -248,7 +248,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
         const float kScaleLog2 = kScale * kLog2e;
         for (int t = 0; t < n_tiles; ++t) {
             if (*abort_flag) break;
-            if (!mbar_wait(&s_full[wg], (uint32_t)(t & 1))) { give_up(); break; }
+            if (!mbar_wait(&s_full[wg], (uint32_t)(t & 1), g.wait_ns)) { give_up(); break; }
             tc_fence_after();
             const int valid = min(kTileKeys, hi - (lo + t * kTileKeys));     // keys of this tile that exist (>= 1)
             const bool full = valid == kTileKeys;
@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
             // So they take turns: B starts the exponentials of tile t when A has issued its own, A those of tile t + 1
             // when B has; each one's wait for the tensor pipe then lies under the other one's exponentials.
             if (kTakeTurns && has_b && (wg == 1 || t > 0)) {
-                if (!mbar_wait(&turn[wg], (uint32_t)((wg == 1 ? t : t - 1) & 1))) { give_up(); break; }
+                if (!mbar_wait(&turn[wg], (uint32_t)((wg == 1 ? t : t - 1) & 1), g.wait_ns)) { give_up(); break; }
             }
             if (t == 0) {
                 // the first tile fixes the reference: a pass for the maximum, then the exponentials
@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
             // rows of V past the valid length may hold anything (even NaN): zero them so that 0 * x stays 0
             if (valid < kTileKeys) {                                // uniform over the CTA (both warpgroups write zeros)
                 const int s = t % kTcStages;
-                if (!mbar_wait(&v_full[s], (uint32_t)((t / kTcStages) & 1))) { give_up(); break; }
+                if (!mbar_wait(&v_full[s], (uint32_t)((t / kTcStages) & 1), g.wait_ns)) { give_up(); break; }
                 uint4 *vrows = reinterpret_cast<uint4 *>(smem + kOffV + s * kTileBytes);
                 for (int e = valid * 8 + wrow; e < kTileKeys * 8; e += 128) vrows[e] = make_uint4(0u, 0u, 0u, 0u);
             }
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
 #pragma unroll
         for (int c = 0; c < kD; ++c) acc[c] = 0.f;
         if (n_tiles > 0 && !*abort_flag) {
-            if (!mbar_wait(&o_final[wg], 0u)) give_up();
+            if (!mbar_wait(&o_final[wg], 0u, g.wait_ns)) give_up();
             else {
                 tc_fence_after();
                 uint32_t ov[2][32];
@@ -366,8 +366,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_attend_tc(Geom g, AttendTcArg
         // tiles that were requested but perhaps never consumed: give every ring slot a bounded chance to land
         for (int s = 0; s < kTcStages && s < n_tiles; ++s) {
             const int t_last = ((n_tiles - 1 - s) / kTcStages) * kTcStages + s;     // the last tile that uses slot s
-            mbar_wait(&k_full[s], (uint32_t)((t_last / kTcStages) & 1));
-            mbar_wait(&v_full[s], (uint32_t)((t_last / kTcStages) & 1));
+            mbar_wait(&k_full[s], (uint32_t)((t_last / kTcStages) & 1), g.wait_ns);
+            mbar_wait(&v_full[s], (uint32_t)((t_last / kTcStages) & 1), g.wait_ns);
         }
     }
     __syncthreads();

@@ -25,6 +25,10 @@ struct Geom {
     const int *u_tab;                     // device [T + 1]: number of selected queries by length
     const int *U_tab;                     // device [T + 1]: number of sampled keys by length
     unsigned *status;                     // device status word
+    unsigned long long wait_ns;           // limit of the bounded device-side waits that take it from here (1 s unless a
+                                          // test shortens it, see psattn_plan_debug_waits)
+    unsigned debug_extra_tx;              // test hook: bytes added to the first expected-bytes count of a kernel's
+                                          // first TMA barrier, so that the barrier never completes and the wait runs out
 };
 
 // Programmatic dependent launch, for kernels that are launched with launch_pdl (psattn_launch.h): lets the
@@ -35,6 +39,27 @@ __device__ __forceinline__ void pdl_enter() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+
+// Phase timing of the fused forward kernel, compiled in only with -DPSATTN_PHASE_STAMPS (a separate build of
+// the library that the benchmark's --phases mode makes and loads; the regular build contains none of it).
+// Called by all threads right after a block-wide barrier; thread 0 adds the time since the CTA's previous stamp
+// to accumulator k (nanoseconds, 64-bit) in the status area of the workspace: bytes [64 + 8 k, 72 + 8 k),
+// k = 1 .. 7; accumulator 0 counts the CTAs.
+#ifdef PSATTN_PHASE_STAMPS
+__device__ __forceinline__ void phase_stamp(const Geom &g, int k) {
+    __shared__ unsigned long long phase_last;
+    if (threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        unsigned long long *acc = reinterpret_cast<unsigned long long *>(g.status) + 8;
+        if (k == 0) atomicAdd(acc, 1ull);
+        else atomicAdd(acc + k, t - phase_last);
+        phase_last = t;
+    }
+}
+#else
+__device__ __forceinline__ void phase_stamp(const Geom &, int) {}
+#endif
 
 __device__ __forceinline__ int seq_len(const Geom &g, int b) {
     if (!g.lengths) return g.T;

@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     if (tid == 32) {
         mbar_init(&P.bar, 1);
         fence_barrier_init();
-        if (L > 0 && !given) measure_issue_keys(smem, &P.bar, &tmKrows, L, b, h, a.pos_t, a.pos_h);
+        if (L > 0 && !given) measure_issue_keys(smem, &P.bar, &tmKrows, L, b, h, a.pos_t, a.pos_h, g.debug_extra_tx);
         tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
     }
     for (int i = tid; i < g.T; i += kFusedThreads) { chosen[i] = 0; if (i >= L) M_s[i] = 0.f; }
@@ -102,6 +102,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     tc_fence_after();
     const uint32_t tmem_base = P.tmem_slot;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    phase_stamp(g, 0);
 
     // ---- steps (a)+(b) ------------------------------------------------------------------------
     bool ok = true;
@@ -109,6 +110,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
         ok = measure_resident<kFusedThreads>(smem, &P.bar, 0u, a.k_bytes, a.stage_bytes, g, unit, b, h, L, U, 0, L, Q,
                                              sidx, M_s);
     __syncthreads();
+    phase_stamp(g, 2);                                         // steps (a)+(b) done (stamp 1: the keys had landed)
     if (M_out != nullptr && !given)
         for (int i = tid; i < g.T; i += kFusedThreads) M_out[(long long)unit * g.T + i] = M_s[i];
 
@@ -140,6 +142,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
         }
     }
     __syncthreads();
+    phase_stamp(g, 3);                                         // step (c) done
 
     // ---- step (d), with the column sums of V riding along ------------------------------------------
     if (ok && L > 0) {
@@ -165,6 +168,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
     }
     tc_fence_before();
     __syncthreads();
+    phase_stamp(g, 4);                                         // step (d) done
 
     // ---- step (e) -----------------------------------------------------------------------------
     {
@@ -183,6 +187,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) k_forward_fused(
         }
     }
     __syncthreads();
+    phase_stamp(g, 5);                                         // step (e) done
     if (warp == 0) tmem_dealloc(tmem_base, kA64TmemCols);
 }
 

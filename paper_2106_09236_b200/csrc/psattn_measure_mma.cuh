@@ -183,11 +183,11 @@ __device__ __forceinline__ void measure_block(const MeasureCtx &cx) {
 // One thread: start the TMA copies of the unit's key rows [0, L) into shared memory at `smem`
 // (row pitch 128 B), all arriving on `bar` (initialised, count 1).  Returns the number of boxes.
 __device__ __forceinline__ int measure_issue_keys(uint8_t *smem, uint64_t *bar, const CUtensorMap *tmK, int L, int b,
-                                                  int h, int pos_t, int pos_h) {
+                                                  int h, int pos_t, int pos_h, uint32_t extra_tx = 0u) {
     using namespace sm100;
     const int n_boxes = (L + kMeasureBoxRows - 1) / kMeasureBoxRows;
     if (n_boxes == 0) return 0;
-    mbar_expect_tx(bar, (uint32_t)n_boxes * kMeasureBoxRows * 128u);
+    mbar_expect_tx(bar, (uint32_t)n_boxes * kMeasureBoxRows * 128u + extra_tx);   // extra_tx: test hook, see Geom
     for (int x = 0; x < n_boxes; ++x) {
         const int key0 = x * kMeasureBoxRows;
         const int c1 = pos_t == 1 ? key0 : (pos_h == 1 ? h : b);
@@ -242,15 +242,16 @@ __device__ __forceinline__ bool measure_resident(uint8_t *smem, uint64_t *bar, u
     for (int blk = 0; blk < kMeasureStages - 1; ++blk) stage_block(blk);
 
     // every thread must take the same branch (both contain barriers): agree on the outcome
-    if (!__syncthreads_and(mbar_wait(bar, bar_phase) ? 1 : 0)) {   // bounded wait expired: report, produce zeros
+    if (!__syncthreads_and(mbar_wait(bar, bar_phase, g.wait_ns) ? 1 : 0)) {   // bounded wait expired: report, produce zeros
         if ((tid & 31) == 0) atomicOr(g.status, kStatusWaitExpired);
         for (int i = q_lo + tid; i < q_end; i += THREADS) out[i] = 0.f;
         cp_async_wait<0>();
         // the bulk copies may still land: do not go on while they can write into this CTA's memory
-        mbar_wait(bar, bar_phase);
+        mbar_wait(bar, bar_phase, g.wait_ns);
         __syncthreads();
         return false;
     }
+    phase_stamp(g, 1);                                    // the unit's keys are in shared memory
     U = min(U, kMeasureMaxU);
     MeasureCtx cx;
     cx.k_base = smem_u32(smem); cx.U = U; cx.L = L; cx.idx_cols = g.idx_cols; cx.status = g.status;

@@ -81,6 +81,7 @@ extern "C" int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, floa
     g.lengths = lengths;
     g.u_tab = nullptr; g.U_tab = nullptr;
     g.status = reinterpret_cast<unsigned *>(scratch);
+    g.wait_ns = 1000ull * 1000ull * 1000ull; g.debug_extra_tx = 0u;
     float *part = scratch + kNoAllocStatusFloats;
     // The array keeps whatever the previous call left.  The partials of this call's units are all
     // rewritten by the column-sum kernel before they are read; only the status word has to start

@@ -46,6 +46,25 @@ def test_two_calls_in_a_row_match_the_planned_entry_point():
         plan.close()
 
 
+def test_second_call_allocates_nothing_and_lengths_are_clamped():
+    """What the entry point is for: once the first call on the device has looked up its scratch array, a call
+    leaves the amount of free device memory exactly as it found it.  Lengths outside [0, T_max] are clamped."""
+    B, H, T = 3, 2, 700
+    V, _, tdt = _case(B, H, T, 3, "bf16", [700, 700, 700])
+    L_bad = torch.tensor([700 + 50, -4, 123], dtype=torch.int32, device="cuda")     # too long, negative, fine
+    got = torch.empty((B, H, 64), dtype=torch.float32, device="cuda")
+    ps.psattn_mean_v_noalloc(V, L_bad, got, B, H, T)            # a first call may do the one-time set-up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    ps.psattn_mean_v_noalloc(V, L_bad, got, B, H, T)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, "the call changed the free device memory"
+    v = V.float().cpu().numpy()
+    want = np.stack([v[0].mean(axis=1), np.zeros((H, 64), dtype=np.float32), v[2, :, :123].mean(axis=1)])
+    assert np.abs(got.cpu().numpy() - want).max() <= 1e-4
+
+
 def test_capacity_and_argument_errors():
     V = torch.zeros((1, 1, 256, 64), dtype=torch.bfloat16, device="cuda")
     out = torch.zeros((1, 1, 64), dtype=torch.float32, device="cuda")
@@ -57,3 +76,6 @@ def test_capacity_and_argument_errors():
     assert ps.psattn_launch_count() == before
     assert lib.psattn_mean_v_noalloc(None, None, out.data_ptr(), 1, 1, 256, 0, None) == 1
     assert lib.psattn_mean_v_noalloc(V.data_ptr(), None, out.data_ptr(), 1, 1, 256, 7, None) == 2
+    # sizes beyond the plan limits are refused before any arithmetic on them
+    assert lib.psattn_mean_v_noalloc(V.data_ptr(), None, out.data_ptr(), 1, 1, 2 ** 31 - 1, 0, None) == 2
+    assert lib.psattn_mean_v_noalloc(V.data_ptr(), None, out.data_ptr(), 2 ** 21, 1, 256, 0, None) == 2

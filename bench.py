@@ -66,12 +66,12 @@ _FUSED_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.
 _STREAM_SOURCES = ["psattn_measure_mma.cu", "psattn_measure_stream.cuh", "psattn_measure_mma.cuh",
                    "psattn_sm100.cuh", "psattn_common.cuh"]
 TRAFFIC = {
-    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53625856, "sources": _FUSED_SOURCES,
+    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53834496, "sources": _FUSED_SOURCES,
                    "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
-                   "sources_sha1": "30622772007f5c0e35b61ed38bfeef9d342cf0d9"},
-    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76343808, "sources": _STREAM_SOURCES,
+                   "sources_sha1": "8beae4c2456c68a3335152a5e1b41121d42337d7"},
+    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76050688, "sources": _STREAM_SOURCES,
                   "profile": "profiles/ncu_full_k_measure_stream_long_bf16.txt",
-                  "sources_sha1": "2cefd328bfe39e8941e1eea3f3e682bc492120bf"},
+                  "sources_sha1": "f298a8beb1a2c3e09ca6e39119780a6b7f509836"},
 }
 
 
@@ -303,7 +303,7 @@ class Ctx:
         return out
 
 
-def gather_probe(cx):
+def gather_probe(cx, full=False):
     """The two gather ceilings of steps (a)+(b), measured here and now with the library's own probe kernels:
     random 128-byte rows out of a chunk resident in shared memory (ldmatrix pattern of the resident-key
     kernel) and out of an L2-resident buffer the size of the keys of `long_bf16` (register loads)."""
@@ -332,6 +332,31 @@ def gather_probe(cx):
     out["l2"] = {"gbs": gbs, "how": "psattn_probe_gather modes 1-2: %d CTAs x 24 warps, 16-byte register loads of random 128-byte "
                                    "rows of a 33.5 MB buffer (L2 resident), best of 5" % cx.sms}
     del buf
+    if not full:
+        return out
+    # the rest of the microbenchmarks (only with --probe gather): what the arithmetic and the index loads of the
+    # measure kernel cost on top of the bare shared-memory gather, and the gather out of the shared memory of a
+    # thread-block cluster
+    names = {3: "shared memory + mma chain (1 round in flight)", 4: "shared memory + mma chains (2 rounds)",
+             5: "shared memory + mma chains (4 rounds)", 6: "shared memory + mma chain + row numbers from a table (1 round)",
+             7: "shared memory + mma chains + row numbers from a table (2 rounds)",
+             8: "shared memory + mma chains + row numbers from a table (4 rounds)"}
+    extra = {}
+    for mode, name in names.items():
+        extra[name] = {"gbs": best(lambda: ps.psattn_probe_gather(mode, None, cx.sms, 16, 4000, sink)), "ctas": cx.sms, "warps": 16}
+    lib = ps.load()
+    import ctypes
+    for cs in (1, 2, 4, 8):
+        ctas = (min(cx.sms, 128) // cs) * cs
+
+        def run(cs=cs, ctas=ctas):
+            rc = lib.psattn_probe_gather(9, None, cs, ctas, 16, 2000, ctypes.c_void_p(sink.data_ptr()),
+                                         ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+            if rc != 0:
+                raise RuntimeError("psattn_probe_gather mode 9 failed: %d" % rc)
+            return ctas * 16 * 2000 * 16
+        extra["distributed shared memory, cluster of %d" % cs] = {"gbs": best(run), "ctas": ctas, "warps": 16}
+    out["more"] = extra
     return out
 
 
@@ -744,7 +769,7 @@ def main():
             print(json.dumps(run_phases(cx, wp)), flush=True)
         return
     cx = Ctx(args)
-    probe = gather_probe(cx)
+    probe = gather_probe(cx, full=args.probe == "gather")
     if args.probe == "gather":
         if cx.rank == 0:
             print(json.dumps({"probe": "gather", "sm_count": cx.sms, "ceilings": probe}), flush=True)

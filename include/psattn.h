@@ -268,6 +268,12 @@ int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, float *vbar, in
  *           global memory / L2 into registers, two rounds in flight per warp (warps_per_cta <= 24;
  *           rounds_per_warp is rounded down to a multiple of the rounds in flight)
  *   mode 2  as mode 1 with four rounds in flight per warp
+ *   mode 3-5 / 6-8  as mode 0 with the arithmetic of the measure kernel behind the loads (a chain of four
+ *           mma.m16n8k16 per round; 1, 2 or 4 rounds interleaved), row numbers from a hash / from a table in shared
+ *           memory (one more 4-byte shared-memory load per lane and round, as in the kernel)
+ *   mode 9 / 10  rows of the shared memory of the CTAs of a thread-block cluster (distributed shared memory),
+ *           read into registers with two / four rounds in flight; n_rows carries the cluster size (1, 2, 4 or 8),
+ *           n_ctas is rounded down to a multiple of it
  * sink: device uint32 (written practically never; it keeps the loads alive). */
 int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_rows, int32_t n_ctas,
                         int32_t warps_per_cta, int32_t rounds_per_warp, uint32_t *sink, void *stream);

@@ -112,6 +112,47 @@ __global__ void __launch_bounds__(1024, 1) k_probe_smem_mma(int rounds, uint32_t
     if (mx + ds == 0.12345f) sink[0] = 1u;
 }
 
+// The same register gather out of the shared memory of the CTAs of a thread-block cluster (distributed shared
+// memory): every CTA holds 1024 rows, a warp reads random rows of random CTAs of its cluster.
+template <int kInFlight>
+__global__ void __launch_bounds__(768, 1) k_probe_dsmem(int rounds, int cluster_size, uint32_t *__restrict__ sink) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int e = tid; e < kProbeSmemRows * 32; e += blockDim.x) reinterpret_cast<uint32_t *>(smem)[e] = (uint32_t)e;
+    // every CTA of the cluster has filled its rows before anybody reads them
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const uint32_t base = sm100::smem_u32(smem);
+    const int g = lane >> 2, t = lane & 3;
+    uint32_t acc = 0;
+    const uint32_t seed = (blockIdx.x * 64u + warp) * 65536u;
+    for (int r0 = 0; r0 + kInFlight <= rounds; r0 += kInFlight) {
+        uint32_t v[kInFlight][4][4];
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const uint32_t hsh = probe_hash(seed + (uint32_t)(r0 + k) * 16u + (uint32_t)(g + 8 * half));
+                const uint32_t row = hsh % kProbeSmemRows, rank = (hsh >> 16) % (uint32_t)cluster_size;
+                uint32_t remote;
+                asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(base + row * 128u + (uint32_t)t * 16u), "r"(rank));
+                asm volatile("ld.shared::cluster.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v[k][2 * half][0]), "=r"(v[k][2 * half][1]), "=r"(v[k][2 * half][2]), "=r"(v[k][2 * half][3]) : "r"(remote));
+                asm volatile("ld.shared::cluster.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v[k][2 * half + 1][0]), "=r"(v[k][2 * half + 1][1]), "=r"(v[k][2 * half + 1][2]), "=r"(v[k][2 * half + 1][3]) : "r"(remote + 64u));
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kInFlight; ++k)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) acc ^= v[k][x][0] ^ v[k][x][1] ^ v[k][x][2] ^ v[k][x][3];
+    }
+    if (acc == 0x12345678u) sink[0] = acc;
+    // nobody leaves while its rows may still be read
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 template <int kInFlight>
 __global__ void __launch_bounds__(768, 1) k_probe_l2(const uint4 *__restrict__ rows, uint32_t n_rows, int rounds,
                                                      uint32_t *__restrict__ sink) {
@@ -179,6 +220,34 @@ extern "C" int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_row
             PSATTN_PROBE_CASE(8, g8, 4, true)
         }
 #undef PSATTN_PROBE_CASE
+    } else if (mode == 9 || mode == 10) {
+        // n_rows carries the cluster size here (1, 2, 4 or 8); n_ctas is rounded down to a multiple of it
+        const int cs = (int)n_rows;
+        if ((cs != 1 && cs != 2 && cs != 4 && cs != 8) || warps_per_cta > 24) return PSATTN_ERR_BAD_DESC;
+        const int ctas = n_ctas / cs * cs;
+        if (ctas < cs) return PSATTN_ERR_BAD_DESC;
+        const size_t smem = (size_t)kProbeSmemRows * 128;
+        static SmemGrant g9, g10;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)ctas);
+        cfg.blockDim = dim3((unsigned)warps_per_cta * 32);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e;
+        if (mode == 9) {
+            if (grant_dynamic_smem(k_probe_dsmem<2>, g9, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+            e = cudaLaunchKernelEx(&cfg, k_probe_dsmem<2>, rounds_per_warp, cs, sink);
+        } else {
+            if (grant_dynamic_smem(k_probe_dsmem<4>, g10, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+            e = cudaLaunchKernelEx(&cfg, k_probe_dsmem<4>, rounds_per_warp, cs, sink);
+        }
+        note_launch();
+        return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? PSATTN_OK : PSATTN_ERR_CUDA;
     } else if (mode == 1 || mode == 2) {
         if (!rows) return PSATTN_ERR_NULL;
         if (n_rows < 1 || n_rows > (1ll << 31) || warps_per_cta > 24) return PSATTN_ERR_BAD_DESC;

@@ -326,6 +326,51 @@ def test_measure_entry_point():
     plan.close()
 
 
+@pytest.mark.parametrize("U_override", [0, 9, 46])
+@pytest.mark.parametrize("T", [1024, 3000])        # keys resident in shared memory / gathered from L2
+def test_measure_with_structured_samples(T, U_override):
+    """Sample rows that are not uniform: every sample in the first 1024 keys, every sample in the last 100
+    keys, one key repeated, a row of equal-score keys (exact zero), ascending runs, an odd and an even sample
+    count, a sequence shorter than T_max whose length is no multiple of any tile; then out-of-range entries,
+    which must be clamped and reported, never followed."""
+    B, H, c = 3, 2, 5.0
+    lengths = [T, T - 37, 129]
+    n_cols = max(orc.count(c, T), U_override)
+    inp = _synth(B, H, T, 700 + T, n_cols, "bf16", lengths)
+    idx = inp["sample_idx"]
+    rng = np.random.default_rng(701)
+    for b, L in enumerate(lengths):
+        idx[b, 0:L:7] = rng.integers(0, min(L, 1024), size=idx[b, 0:L:7].shape)        # all in the first chunk
+        idx[b, 1:L:7] = rng.integers(max(0, L - 100), L, size=idx[b, 1:L:7].shape)      # all at the end
+        idx[b, 2:L:7] = rng.integers(0, L, size=(len(range(2, L, 7)), 1))               # one key, repeated
+        idx[b, 3:L:7] = np.sort(idx[b, 3:L:7], axis=-1)                                 # ascending
+    inp["K"][0, :, 5:9] = inp["K"][0, :, 5:6]                                           # four identical key rows
+    idx[0, 11] = np.resize(np.array([5, 6, 7, 8], dtype=np.int32), n_cols)              # -> constant scores
+    dev, tdt = _dev(inp, "bf16")
+    plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n_cols, U_override=U_override)
+    M = plan.psattn_measure(dev["Q"], dev["K"], dev["lengths"], dev["sample_idx"])
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() == 0
+    Mh = M.cpu().numpy()
+    parity.check_measure(Mh, orc.measure(inp["Q"], inp["K"], idx, inp["lengths"], c=c, U_override=U_override),
+                         inp["lengths"])
+    assert np.all(Mh[0, :, 11] == 0.0) and np.all(Mh[:, :, 2][:, :] == 0.0)           # constant scores: exactly zero
+    assert Mh.min() >= 0.0
+    # out-of-range entries: clamped into [0, len), status bit 0, no fault
+    bad = idx.copy()
+    bad[1, 40, 0] = T + 12345
+    bad[2, 3, 1] = -7
+    M2 = plan.psattn_measure(dev["Q"], dev["K"], dev["lengths"], torch.from_numpy(bad).cuda())
+    torch.cuda.synchronize()
+    assert plan.psattn_read_status() & 1
+    clamped = bad.copy()
+    clamped[1, 40, 0] = lengths[1] - 1
+    clamped[2, 3, 1] = 0
+    parity.check_measure(M2.cpu().numpy(), orc.measure(inp["Q"], inp["K"], clamped, inp["lengths"], c=c,
+                                                       U_override=U_override), inp["lengths"])
+    plan.close()
+
+
 def test_measure_per_head_samples():
     B, H, T, c = 2, 3, 70, 5.0
     n = orc.count(c, T)

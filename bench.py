@@ -738,6 +738,51 @@ def run_phases(cx, w):
     return out
 
 
+def run_timeline(cx, w):
+    """Begin and end of every kernel of the staged schedule inside one CUDA-graph replay of psattn_forward: the same
+    stamped build records, per kernel, when its first block got past the wait for the grid before it and when its
+    last block ended.  One replay at a time with an idle device before it, so the absolute times are those of a
+    cold start (a few us above the step time of back-to-back replays); the order and the gaps are what to read."""
+    torch, ps = cx.torch, cx.ps
+    tdt, elem = torch.bfloat16, 2
+    n_cols = max(ps.psattn_count(w.c, L) for L in range(1, w.T + 1))
+    plan = ps.Plan(w.B, w.H, w.T, dtype=tdt, c=w.c, idx_cols=n_cols)
+    sets, _, _ = make_sets(cx, w, n_cols, plan, tdt, elem)
+
+    def step(s):
+        d = sets[s]
+        plan.psattn_forward(d["Q"], d["K"], d["V"], d["lengths"], d["sample_idx"], d["O"], d["sel"])
+    rp = Replay(cx, step, len(sets), use_graph=True)
+    for k in range(3 * len(sets)):
+        rp(k)
+    torch.cuda.synchronize()
+    slots = plan.workspace[128:256].view(torch.int64)
+    init = torch.tensor([2 ** 62, 0] * 8, dtype=torch.int64, device="cuda")
+    names = ["k_measure_stream", "k_select_slice", "k_select_merge", "k_attend64", "k_attend_combine",
+             "k_colsum (side stream)", "k_select: mean(V) from the partials (side stream)", "k_fill (side stream)"]
+    runs = []
+    for rep in range(5):
+        slots.copy_(init)
+        torch.cuda.synchronize()
+        rp(rep)
+        torch.cuda.synchronize()
+        a = slots.cpu().numpy().reshape(8, 2)
+        used = [k for k in range(8) if a[k, 1] > 0]
+        t0 = min(a[k, 0] for k in used)
+        runs.append({names[k]: [round(float(a[k, 0] - t0) / 1e3, 2), round(float(a[k, 1] - t0) / 1e3, 2)] for k in used})
+    med = {}
+    for name in runs[0]:
+        if all(name in r for r in runs):
+            med[name] = [float(np.median([r[name][0] for r in runs])), float(np.median([r[name][1] for r in runs]))]
+    order = sorted(med, key=lambda nm: med[nm][0])
+    out = {"timeline": "kernels of one graph replay of psattn_forward, us from the first kernel's begin: "
+                       "[first block released, last block ended], median of %d single replays" % len(runs),
+           "workload": w.name, "kernels": {nm: med[nm] for nm in order},
+           "note": "stamps cost two atomics per block; the step time of the regular build is the one bench.py reports"}
+    plan.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -748,7 +793,8 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "staged", "fused"])
     ap.add_argument("--probe", default=None, choices=["gather"], help="run only the named microbenchmark")
     ap.add_argument("--phases", action="store_true",
-                    help="per-phase times of the fused forward kernel (builds a stamped copy of the library first)")
+                    help="per-phase times of the fused forward kernel and begin/end of the kernels of the staged "
+                         "schedule (builds a stamped copy of the library first)")
     ap.add_argument("--no-graph", action="store_true", help="time direct calls instead of CUDA-graph replays")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle timing")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense comparator timing")
@@ -764,9 +810,11 @@ def main():
         from paper_2106_09236_b200 import build as lib_build
         os.environ["PSATTN_LIBRARY"] = lib_build.build(phase_stamps=True)
         cx = Ctx(args)
-        wp = w if w.name != HEADLINE else wl.WORKLOADS[OTHER]          # the fused kernel takes T_max <= ~1100
         if cx.rank == 0:
-            print(json.dumps(run_phases(cx, wp)), flush=True)
+            # the fused kernel takes T_max <= ~1100: its phases on the shorter workload, the kernels of the staged
+            # schedule on the longer one
+            for wp in (w, wl.WORKLOADS[OTHER if w.name == HEADLINE else HEADLINE]):
+                print(json.dumps(run_timeline(cx, wp) if wp.T > 1100 else run_phases(cx, wp)), flush=True)
         return
     cx = Ctx(args)
     probe = gather_probe(cx, full=args.probe == "gather")

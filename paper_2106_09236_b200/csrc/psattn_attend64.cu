@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(kA64Threads, 1) k_attend64(Geom g, Attend64Arg
     // columns before a CTA of this grid had allocated, that CTA would block in tcgen05.alloc for good.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");                // nothing above touches global data
+    KernelSpan span(g, kKernelAttend64);
 
     Attend64Job j;
     j.b = unit / g.H; j.h = unit % g.H; j.L = seq_len(g, j.b);

@@ -61,6 +61,28 @@ __device__ __forceinline__ void phase_stamp(const Geom &g, int k) {
 __device__ __forceinline__ void phase_stamp(const Geom &, int) {}
 #endif
 
+// Begin and end of a kernel of the staged schedule, same build only: the earliest moment a block got past its
+// wait for the grid before it and the latest moment a block ended (%globaltimer, nanoseconds), in the status area at
+// bytes [128 + 16 k, 144 + 16 k), k = which kernel (KernelId).  The host sets begin to a large value and end to 0.
+enum KernelId { kKernelMeasure = 0, kKernelSelectSlice, kKernelSelectMerge, kKernelAttend64, kKernelCombine, kKernelColsum,
+                kKernelSelect, kKernelFill };
+#ifdef PSATTN_PHASE_STAMPS
+struct KernelSpan {
+    unsigned long long *slot;
+    __device__ __forceinline__ KernelSpan(const Geom &g, int k) {
+        slot = reinterpret_cast<unsigned long long *>(g.status) + 16 + 2 * k;
+        if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); atomicMin(slot, t); }
+    }
+    __device__ __forceinline__ ~KernelSpan() {
+        if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); atomicMax(slot + 1, t); }
+    }
+};
+#else
+struct KernelSpan {
+    __device__ __forceinline__ KernelSpan(const Geom &, int) {}
+};
+#endif
+
 __device__ __forceinline__ int seq_len(const Geom &g, int b) {
     if (!g.lengths) return g.T;
     int L = g.lengths[b];

@@ -60,6 +60,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) k_measure_stream(Geom g, in
     const int unit = blockIdx.x / q_slices, slice = blockIdx.x % q_slices;
     const int b = unit / g.H, h = unit % g.H;
     pdl_enter();
+    KernelSpan span(g, kKernelMeasure);
     const int L = seq_len(g, b);
     const int U = min(g.U_tab[L], g.idx_cols);
     // slices in whole staged blocks so that every CTA but the last works on full blocks

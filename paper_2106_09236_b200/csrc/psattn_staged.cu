@@ -97,6 +97,7 @@ __global__ void __launch_bounds__(256) k_colsum(Geom g, const DT *__restrict__ V
     const int unit = blockIdx.x, chunk = blockIdx.y;
     const int b = unit / g.H, h = unit % g.H;
     pdl_enter();
+    KernelSpan span(g, kKernelColsum);
     const int L = seq_len(g, b);
     const int sub = threadIdx.x & 7, r0 = threadIdx.x >> 3;
     const int lo = chunk * kColsumRows, hi = min(L, lo + kColsumRows);
@@ -133,6 +134,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_select(Geom g, const float *
     const int unit = blockIdx.x;
     const int b = unit / g.H;
     pdl_enter();
+    KernelSpan span(g, kKernelSelect);
     const int L = seq_len(g, b);
     const int u = min(min(g.u_tab[L], g.u_max), L);
     const float *Mu = M + (long long)unit * g.T;
@@ -171,6 +173,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_select_slice(Geom g, const f
     const int unit = blockIdx.x / slices, sl = blockIdx.x % slices;
     const int b = unit / g.H;
     pdl_enter();
+    KernelSpan span(g, kKernelSelectSlice);
     const int L = seq_len(g, b);
     const int u = min(min(g.u_tab[L], g.u_max), L);
     const int lo = sl * width, n = max(0, min(L - lo, width));
@@ -193,6 +196,7 @@ __global__ void __launch_bounds__(256) k_select_merge(Geom g, const float *__res
     const int unit = blockIdx.x;
     const int b = unit / g.H;
     pdl_enter();
+    KernelSpan span(g, kKernelSelectMerge);
     const int L = seq_len(g, b);
     const int u = min(min(g.u_tab[L], g.u_max), L);
     const int n = slices * g.u_max;                            // candidate slots, -1 padded per range
@@ -323,6 +327,7 @@ __global__ void __launch_bounds__(256) k_attend_combine(Geom g, const int *__res
                                                         int out_by_position, float *__restrict__ vbar) {
     const int n_slots = n_rows + (vbar ? 1 : 0);           // slot n_rows (if any) is the all-ones row
     pdl_enter();
+    KernelSpan span(g, kKernelCombine);
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long rowid = t / kD;
     const int c = (int)(t % kD);
@@ -376,6 +381,7 @@ __global__ void __launch_bounds__(256) k_fill(Geom g, const DT *__restrict__ V,
     const int unit = blockIdx.x;
     const int b = unit / g.H, h = unit % g.H;
     pdl_enter();
+    KernelSpan span(g, kKernelFill);
     const int L = seq_len(g, b);
     const int lo = blockIdx.y * kFillRows;
     for (int t = threadIdx.x; t < kFillRows; t += blockDim.x) chosen[t] = 0;

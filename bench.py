@@ -700,9 +700,18 @@ def run_dense(cx, w, r):
     d_ms = float(np.median(reps))
     flops = 4.0 * w.d * sum(int(L) * int(L) for L in r["host0"]["lengths"]) * w.H
     tp = tensor_peak()
+    # With d_head = 64 dense attention is bound by its exponentials before its matrix products: one per score, and the
+    # special-function units of an SM deliver 16 per clock (4 per sub-partition), against 4 * 64 flops per score.
+    mhz = (r["clocks"] or {}).get("sm_mhz") or (r["clocks"] or {}).get("sm_max_mhz") or 1965.0
+    exps = float(sum(int(L) * int(L) for L in r["host0"]["lengths"]) * w.H)
+    exp_floor_ms = exps / (16.0 * cx.sms * mhz * 1e6) * 1e3
     return {"ms_per_step": d_ms, "repeats": len(reps), "speedup_sparse_vs_dense": d_ms / r["ms"],
             "tflops": flops / (d_ms * 1e-3) / 1e12, "frac_of_tensor_peak": flops / (d_ms * 1e-3) / 1e12 / tp[0],
-            "peak_kind": "of " + tp[1], "workspace_bytes_sparse": plan.workspace_bytes,
+            "peak_kind": "of " + tp[1],
+            "roofline_exp": {"bound": "alu", "unit": "exp/s", "exps_per_step": exps, "achieved": exps / (d_ms * 1e-3),
+                             "peak": 16.0 * cx.sms * mhz * 1e6, "frac": exp_floor_ms / d_ms, "floor_ms": exp_floor_ms,
+                             "peak_kind": "16 exponentials per clock and SM x %d SMs x %.0f MHz (median SM clock of this run)" % (cx.sms, mhz)},
+            "workspace_bytes_sparse": plan.workspace_bytes,
             "score_matrix_bytes_if_materialised": 4 * w.B * w.H * w.T * w.T}
 
 

@@ -356,6 +356,12 @@ def gather_probe(cx, full=False):
                 raise RuntimeError("psattn_probe_gather mode 9 failed: %d" % rc)
             return ctas * 16 * 2000 * 16
         extra["distributed shared memory, cluster of %d" % cs] = {"gbs": best(run), "ctas": ctas, "warps": 16}
+    # the same L2 gather through the copy engine (one 128-byte bulk copy per row), alone and beside register loads
+    buf = torch.randn(int(33.5e6 / 4), device="cuda")
+    for mode, name in ((11, "L2 through 128-byte bulk copies into shared memory"),
+                       (12, "L2, every sixth warp with bulk copies beside register loads")):
+        extra[name] = {"gbs": best(lambda: ps.psattn_probe_gather(mode, buf, cx.sms, 24, 800, sink)), "ctas": cx.sms, "warps": 24}
+    del buf
     out["more"] = extra
     return out
 

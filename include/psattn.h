@@ -274,7 +274,13 @@ int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, float *vbar, in
  *   mode 9 / 10  rows of the shared memory of the CTAs of a thread-block cluster (distributed shared memory),
  *           read into registers with two / four rounds in flight; n_rows carries the cluster size (1, 2, 4 or 8),
  *           n_ctas is rounded down to a multiple of it
- * sink: device uint32 (written practically never; it keeps the loads alive). */
+ *   mode 11 as mode 1 through the copy engine: one 128-byte bulk copy per row into a ring in shared memory, two rounds
+ *           in flight per warp (rounds_per_warp is rounded down to a multiple of 4)
+ *   mode 12 mode 11 and mode 1 in one kernel: every sixth warp uses bulk copies, for half as many rounds; the others
+ *           register loads.  It gathers n_ctas * (w - b + b / 2) * rounds * 16 rows, b = the warps among the
+ *           warps_per_cta = w whose number is 5 modulo 6.
+ * sink: device uint32[2] (written practically never; it keeps the loads alive; sink[1] = 0xdead if a bounded wait of
+ * mode 11 / 12 ran out). */
 int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_rows, int32_t n_ctas,
                         int32_t warps_per_cta, int32_t rounds_per_warp, uint32_t *sink, void *stream);
 

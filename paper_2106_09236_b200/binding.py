@@ -141,8 +141,12 @@ def psattn_probe_gather(mode, rows, n_ctas, warps_per_cta, rounds_per_warp, sink
     n_rows = 0 if rows is None else rows.numel() * rows.element_size() // 128
     _check(load().psattn_probe_gather(int(mode), _ptr(rows), n_rows, int(n_ctas), int(warps_per_cta),
                                       int(rounds_per_warp), _ptr(sink), _stream()))
-    per = {0: 1, 1: 2, 2: 4, 3: 1, 4: 2, 5: 4, 6: 1, 7: 2, 8: 4}[int(mode)]       # rounds in flight: the count is a multiple
-    return int(n_ctas) * int(warps_per_cta) * (int(rounds_per_warp) // per * per) * 16
+    per = {0: 1, 1: 2, 2: 4, 3: 1, 4: 2, 5: 4, 6: 1, 7: 2, 8: 4, 11: 4, 12: 4}[int(mode)]   # the round count is a multiple of this
+    rounds = int(rounds_per_warp) // per * per
+    if int(mode) == 12:                                     # every sixth warp takes half as many rounds
+        n_bulk = len([w for w in range(int(warps_per_cta)) if w % 6 == 5])
+        return int(n_ctas) * ((int(warps_per_cta) - n_bulk) * rounds + n_bulk * (rounds // 2)) * 16
+    return int(n_ctas) * int(warps_per_cta) * rounds * 16
 
 
 class Plan:

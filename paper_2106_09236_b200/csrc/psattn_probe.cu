@@ -185,6 +185,79 @@ __global__ void __launch_bounds__(768, 1) k_probe_l2(const uint4 *__restrict__ r
     if (acc == 0x12345678u) sink[0] = acc;
 }
 
+
+// The L2 gather through the copy engine instead of the load/store unit: lanes 0-15 of a warp each ask for one row
+// with a 128-byte bulk copy into the warp's ring in shared memory (one mbarrier per ring slot counts the bytes), two
+// rounds in flight.  MIXED: only every sixth warp does so, with half as many rounds; the others read their rows with
+// 16-byte register loads as k_probe_l2 - does the copy engine add to what the load/store unit gets out of L2?
+template <bool MIXED>
+__global__ void __launch_bounds__(768, 1) k_probe_bulk(const uint4 *__restrict__ rows, uint32_t n_rows, int rounds,
+                                                       uint32_t *__restrict__ sink) {
+    constexpr int kInFlight = 2;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nw = blockDim.x >> 5;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)nw * kInFlight * 2048);
+    if (lane == 0)
+        for (int s = 0; s < kInFlight; ++s) sm100::mbar_init(&bars[warp * kInFlight + s], 1);
+    sm100::fence_barrier_init();
+    __syncthreads();
+    const uint32_t seed = (blockIdx.x * 64u + warp) * 65536u;
+    uint32_t acc = 0;
+    if (MIXED && (warp % 6) != 5) {
+        const int g = lane >> 2, t = lane & 3;
+        for (int r0 = 0; r0 < rounds; r0 += kInFlight) {
+            uint4 v[kInFlight][4];
+#pragma unroll
+            for (int k = 0; k < kInFlight; ++k) {
+                const uint32_t ra = probe_hash(seed + (uint32_t)(r0 + k) * 16u + (uint32_t)g) % n_rows;
+                const uint32_t rb = probe_hash(seed + (uint32_t)(r0 + k) * 16u + (uint32_t)(g + 8)) % n_rows;
+                const uint4 *pa = rows + (size_t)ra * 8 + t, *pb = rows + (size_t)rb * 8 + t;
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v[k][0].x), "=r"(v[k][0].y), "=r"(v[k][0].z), "=r"(v[k][0].w) : "l"(pa));
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v[k][1].x), "=r"(v[k][1].y), "=r"(v[k][1].z), "=r"(v[k][1].w) : "l"(pa + 4));
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v[k][2].x), "=r"(v[k][2].y), "=r"(v[k][2].z), "=r"(v[k][2].w) : "l"(pb));
+                asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v[k][3].x), "=r"(v[k][3].y), "=r"(v[k][3].z), "=r"(v[k][3].w) : "l"(pb + 4));
+            }
+#pragma unroll
+            for (int k = 0; k < kInFlight; ++k)
+#pragma unroll
+                for (int x = 0; x < 4; ++x) acc ^= v[k][x].x ^ v[k][x].y ^ v[k][x].z ^ v[k][x].w;
+        }
+    } else {
+        if (MIXED) rounds /= 2;
+        uint8_t *ring = smem + (size_t)warp * kInFlight * 2048;
+        uint64_t *bar = &bars[warp * kInFlight];
+        auto issue = [&](int r) {
+            const int s = r % kInFlight;
+            if (lane == 0) sm100::mbar_expect_tx(&bar[s], 2048);
+            __syncwarp();
+            if (lane < 16) {
+                const uint32_t row = probe_hash(seed + (uint32_t)r * 16u + (uint32_t)lane) % n_rows;
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 128, [%2];"
+                             ::"r"(sm100::smem_u32(ring + s * 2048 + lane * 128)), "l"(rows + (size_t)row * 8),
+                               "r"(sm100::smem_u32(&bar[s])) : "memory");
+            }
+        };
+        for (int r = 0; r < kInFlight && r < rounds; ++r) issue(r);
+        bool ok = true;
+        for (int r = 0; r < rounds && ok; ++r) {
+            const int s = r % kInFlight;
+            ok = sm100::mbar_wait(&bar[s], (uint32_t)((r / kInFlight) & 1));     // bounded
+            acc ^= *reinterpret_cast<const uint32_t *>(ring + s * 2048 + lane * 64);
+            __syncwarp();
+            if (ok && r + kInFlight < rounds) issue(r + kInFlight);
+        }
+        if (!ok) {                                             // give the copies in flight a bounded chance to land
+            for (int s = 0; s < kInFlight; ++s) sm100::mbar_wait(&bar[s], 0);
+            sink[1] = 0xdeadu;
+        }
+    }
+    if (acc == 0x12345678u) sink[0] = acc;
+}
+
 }  // namespace psattn
 
 using namespace psattn;
@@ -248,6 +321,20 @@ extern "C" int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_row
         }
         note_launch();
         return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? PSATTN_OK : PSATTN_ERR_CUDA;
+    } else if (mode == 11 || mode == 12) {
+        if (!rows) return PSATTN_ERR_NULL;
+        if (n_rows < 1 || n_rows > (1ll << 31) || warps_per_cta > 24) return PSATTN_ERR_BAD_DESC;
+        if ((reinterpret_cast<uintptr_t>(rows) & 15u) != 0) return PSATTN_ERR_MISALIGNED;
+        const size_t smem = (size_t)warps_per_cta * 2 * 2048 + (size_t)warps_per_cta * 2 * 8 + 64;
+        static SmemGrant g11, g12;
+        const dim3 grid((unsigned)n_ctas), block((unsigned)warps_per_cta * 32);
+        if (mode == 11) {
+            if (grant_dynamic_smem(k_probe_bulk<false>, g11, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+            k_probe_bulk<false><<<grid, block, smem, st>>>((const uint4 *)rows, (uint32_t)n_rows, rounds_per_warp / 4 * 4, sink);
+        } else {
+            if (grant_dynamic_smem(k_probe_bulk<true>, g12, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+            k_probe_bulk<true><<<grid, block, smem, st>>>((const uint4 *)rows, (uint32_t)n_rows, rounds_per_warp / 4 * 4, sink);
+        }
     } else if (mode == 1 || mode == 2) {
         if (!rows) return PSATTN_ERR_NULL;
         if (n_rows < 1 || n_rows > (1ll << 31) || warps_per_cta > 24) return PSATTN_ERR_BAD_DESC;

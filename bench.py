@@ -361,6 +361,21 @@ def gather_probe(cx, full=False):
     for mode, name in ((11, "L2 through 128-byte bulk copies into shared memory"),
                        (12, "L2, every sixth warp with bulk copies beside register loads")):
         extra[name] = {"gbs": best(lambda: ps.psattn_probe_gather(mode, buf, cx.sms, 24, 800, sink)), "ctas": cx.sms, "warps": 24}
+    # the inner loop of a chunk-resident form of the long-sequence kernel (keys of a 1024-key chunk in shared memory, the
+    # samples bucketed by chunk): useful rows per second, to set against what the L2-gather kernel achieves
+    for mode, name in ((13, "chunk-resident bucketed loop, independent counts (useful rows)"),
+                       (14, "chunk-resident bucketed loop, counts sorted within 128-query blocks (useful rows)")):
+        def run(mode=mode):
+            sink.zero_()
+            rc = lib.psattn_probe_gather(mode, ctypes.c_void_p(buf.data_ptr()), buf.numel() * 4 // 128, cx.sms, 16, 8,
+                                         ctypes.c_void_p(sink.data_ptr()), ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+            if rc != 0:
+                raise RuntimeError("psattn_probe_gather mode %d failed: %d" % (mode, rc))
+            return cx.sms * 8 * 2048 * 46 // 8            # expected pairs (the kernel's own count is in sink[2..3])
+        gbs = best(run)
+        pairs = int(sink[2:4].view(torch.int64).item())
+        extra[name] = {"gbs": gbs * pairs / (cx.sms * 8 * 2048 * 46 // 8), "ctas": cx.sms, "warps": 16,
+                       "pairs_per_query_and_chunk": pairs / float(cx.sms * 8 * 2048)}
     del buf
     out["more"] = extra
     return out

@@ -279,8 +279,16 @@ int psattn_mean_v_noalloc(const void *V, const int32_t *lengths, float *vbar, in
  *   mode 12 mode 11 and mode 1 in one kernel: every sixth warp uses bulk copies, for half as many rounds; the others
  *           register loads.  It gathers n_ctas * (w - b + b / 2) * rounds * 16 rows, b = the warps among the
  *           warps_per_cta = w whose number is 5 modulo 6.
- * sink: device uint32[2] (written practically never; it keeps the loads alive; sink[1] = 0xdead if a bounded wait of
- * mode 11 / 12 ran out). */
+ *   mode 13 / 14  the inner loop of a chunk-resident form of steps (a)+(b) for long sequences: per work item a 1024-row
+ *           chunk of `rows` is copied into shared memory and 2048 queries gather from it the samples that fall into it
+ *           (Binomial(46, 1/8) of them per query; a warp's eight queries advance together, two rows per query and
+ *           round), their own rows staged through shared memory.  Mode 13: independent counts; mode 14: the counts of
+ *           a warp's eight queries are neighbours in the sorted order of a 128-query block.  n_ctas CTAs of 16 warps
+ *           (warps_per_cta must be 16), rounds_per_warp = work items per CTA; n_rows >= 4096.  The number of useful
+ *           (query, key) pairs is ADDED to the 64-bit counter at sink[2..3] (zero it before the launch; sink 8-byte
+ *           aligned).
+ * sink: device uint32[4] (sink[0] is written practically never; it keeps the loads alive; sink[1] = 0xdead if a bounded
+ * wait of mode 11 / 12 ran out). */
 int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_rows, int32_t n_ctas,
                         int32_t warps_per_cta, int32_t rounds_per_warp, uint32_t *sink, void *stream);
 

@@ -9,6 +9,7 @@
 #include "../../include/psattn.h"
 
 #include "psattn_launch.h"
+#include <cmath>
 #include "psattn_sm100.cuh"
 
 namespace psattn {
@@ -258,6 +259,106 @@ __global__ void __launch_bounds__(768, 1) k_probe_bulk(const uint4 *__restrict__
     if (acc == 0x12345678u) sink[0] = acc;
 }
 
+
+// What a chunk-resident form of steps (a)+(b) could reach for long sequences: a 1024-key chunk (128 KB) sits in shared
+// memory, and the (query, sampled key) pairs whose key lies in the chunk are gathered from there.  A query has
+// Binomial(U, 1/8) samples in one of eight chunks; the mma layout gives each of a warp's eight queries two rows per
+// round, so a group of eight costs max over its queries of ceil(n / 2) rounds.  Per work item (one chunk, 2048
+// queries): the chunk is copied in, then every warp takes groups of eight queries - their rows of Q staged through
+// shared memory (cp.async, one group ahead) and read as mma fragments, their row numbers read from a table, the rounds
+// as in k_probe_smem_mma.  kSorted: the counts of a group are neighbours in the sorted order of their 128-query block
+// (what a pre-pass that orders the queries of a block by count would deliver); otherwise they are independent draws.
+// counts: 128 quantiles of the count distribution.  The kernel adds the useful pairs to sink[2..3] (64 bit).
+struct ProbeCounts { unsigned char q[128]; };
+
+template <bool kSorted>
+__global__ void __launch_bounds__(512, 1) k_probe_bucketed(const uint4 *__restrict__ rows, uint32_t n_rows, int items,
+                                                           ProbeCounts counts, uint32_t *__restrict__ sink) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    constexpr int kQueries = 2048;
+    uint8_t *qstage = smem + kProbeSmemRows * 128;                       // [16 warps][2][1 KB]
+    uint32_t *table = reinterpret_cast<uint32_t *>(qstage + 16 * 2 * 1024);   // 4096 row numbers
+    unsigned char *cnt = reinterpret_cast<unsigned char *>(table + 4096);     // counts of the item's queries
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int e = tid; e < 4096; e += blockDim.x) table[e] = probe_hash((uint32_t)e * 7919u + blockIdx.x) % kProbeSmemRows;
+    const uint32_t base = sm100::smem_u32(smem), tbase = sm100::smem_u32(table);
+    const int l7 = lane & 7;
+    uint32_t off[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) off[t] = (uint32_t)((2 * t + (lane >> 4) + l7) & 7) << 4;
+    const uint32_t slot = (uint32_t)(l7 + 8 * ((lane >> 3) & 1));
+    float mx = 0.f, ds = 0.f;
+    unsigned long long pairs = 0;
+    for (int item = 0; item < items; ++item) {
+        const uint32_t work = (uint32_t)(blockIdx.x * items + item);
+        __syncthreads();                                                 // everybody has left the chunk of the item before
+        // the chunk: 1024 consecutive rows
+        const uint32_t c0 = (work * 1024u) % (n_rows - 1024u);
+        for (int e = tid; e < kProbeSmemRows * 8; e += blockDim.x) reinterpret_cast<uint4 *>(smem)[e] = __ldg(rows + (size_t)c0 * 8 + e);
+        for (int q = tid; q < kQueries; q += blockDim.x)
+            cnt[q] = kSorted ? counts.q[q & 127] : counts.q[probe_hash(work * 4096u + (uint32_t)q) & 127];
+        __syncthreads();
+        const uint32_t q0 = (work * 2048u + 12345u) % (n_rows - 2048u);  // the item's rows of Q, consecutive
+        uint8_t *st = qstage + warp * 2048;
+        auto stage_q = [&](int grp, int buf) {                           // 8 rows x 128 B: two 16-byte pieces per lane
+            const uint4 *src = rows + (size_t)(q0 + grp * 8) * 8;
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {                                // piece c of row r goes to place (c + r) mod 8 of the row
+                const int pc = lane + 32 * x, r = pc >> 3, c = pc & 7;
+                const uint32_t dst = sm100::smem_u32(st + buf * 1024) + (uint32_t)(r * 128 + (((c + r) & 7) << 4));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src + pc) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        int it = 0;
+        stage_q(warp, 0);
+        for (int grp = warp; grp < kQueries / 8; grp += 16, ++it) {
+            if (grp + 16 < kQueries / 8) { stage_q(grp + 16, (it + 1) & 1); asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+            uint32_t bq[8];
+            const uint32_t qa = sm100::smem_u32(st + (it & 1) * 1024) + (uint32_t)l7 * 128u;
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(bq[0]), "=r"(bq[1]), "=r"(bq[2]), "=r"(bq[3]) : "r"(qa + (uint32_t)((((lane >> 3) + l7) & 7) << 4)));
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(bq[4]), "=r"(bq[5]), "=r"(bq[6]), "=r"(bq[7]) : "r"(qa + (uint32_t)((((lane >> 3) + 4 + l7) & 7) << 4)));
+            int n = cnt[grp * 8 + l7];                                   // lanes with the same l7 agree
+            int rounds = (n + 1) >> 1;
+#pragma unroll
+            for (int o = 1; o < 8; o <<= 1) rounds = max(rounds, __shfl_xor_sync(0xffffffffu, rounds, o));
+            if (lane < 8) pairs += (unsigned long long)n;
+            for (int r = 0; r < rounds; ++r) {
+                uint32_t row;
+                const uint32_t ta = tbase + ((((uint32_t)(it * 16 + r) * 16u + slot + (uint32_t)warp * 64u) & 4095u) << 2);
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(row) : "r"(ta));
+                const uint32_t ra = base + row * 128u;
+                float c[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    uint32_t a0, a1, a2, a3;
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(ra + off[t]));
+                    if (t == 0)
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%10, %10, %10, %10};"
+                                     : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bq[0]), "r"(bq[1]), "f"(0.f));
+                    else
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(bq[2 * t]), "r"(bq[2 * t + 1]));
+                }
+                mx = fmaxf(mx, fmaxf(c[0], c[2]));
+                ds += c[1] + c[3];
+            }
+            __syncwarp();
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) pairs += __shfl_xor_sync(0xffffffffu, pairs, o);
+    if (lane == 0) atomicAdd(reinterpret_cast<unsigned long long *>(sink + 2), pairs);
+    if (mx + ds == 0.12345f) sink[0] = 1u;
+}
+
 }  // namespace psattn
 
 using namespace psattn;
@@ -334,6 +435,37 @@ extern "C" int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_row
         } else {
             if (grant_dynamic_smem(k_probe_bulk<true>, g12, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
             k_probe_bulk<true><<<grid, block, smem, st>>>((const uint4 *)rows, (uint32_t)n_rows, rounds_per_warp / 4 * 4, sink);
+        }
+    } else if (mode == 13 || mode == 14) {
+        if (!rows) return PSATTN_ERR_NULL;
+        if (n_rows < 4096 || n_rows > (1ll << 31) || warps_per_cta != 16) return PSATTN_ERR_BAD_DESC;
+        if ((reinterpret_cast<uintptr_t>(rows) & 15u) != 0 || (reinterpret_cast<uintptr_t>(sink) & 7u) != 0) return PSATTN_ERR_MISALIGNED;
+        // 128 quantiles of Binomial(46, 1/8): the number of a query's 46 samples that fall into one of eight chunks
+        ProbeCounts pc;
+        {
+            double pmf[47], cdf = 0.0;
+            for (int k = 0; k <= 46; ++k) {
+                double c = 1.0;
+                for (int j = 0; j < k; ++j) c = c * (46 - j) / (j + 1);
+                pmf[k] = c * std::pow(0.125, k) * std::pow(0.875, 46 - k);
+            }
+            int k = 0;
+            cdf = pmf[0];
+            for (int i = 0; i < 128; ++i) {
+                const double u = (i + 0.5) / 128.0;
+                while (cdf < u && k < 46) cdf += pmf[++k];
+                pc.q[i] = (unsigned char)k;
+            }
+        }
+        const size_t smem = (size_t)kProbeSmemRows * 128 + 16 * 2 * 1024 + 4096 * 4 + 2048;
+        static SmemGrant g13, g14;
+        const dim3 grid((unsigned)n_ctas), block(512);
+        if (mode == 13) {
+            if (grant_dynamic_smem(k_probe_bucketed<false>, g13, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+            k_probe_bucketed<false><<<grid, block, smem, st>>>((const uint4 *)rows, (uint32_t)n_rows, rounds_per_warp, pc, sink);
+        } else {
+            if (grant_dynamic_smem(k_probe_bucketed<true>, g14, smem) != cudaSuccess) return PSATTN_ERR_CUDA;
+            k_probe_bucketed<true><<<grid, block, smem, st>>>((const uint4 *)rows, (uint32_t)n_rows, rounds_per_warp, pc, sink);
         }
     } else if (mode == 1 || mode == 2) {
         if (!rows) return PSATTN_ERR_NULL;

@@ -22,6 +22,21 @@ def test_every_mode_runs_on_a_small_buffer():
     torch.cuda.synchronize()
 
 
+def test_bucketed_chunk_loop_counts_its_pairs():
+    lib = ps.load()
+    sink = torch.zeros(4, dtype=torch.int32, device="cuda")
+    rows = torch.randn(8192 * 32, device="cuda")                # 8192 rows of 128 bytes
+    for mode in (13, 14):
+        sink.zero_()
+        assert lib.psattn_probe_gather(mode, rows.data_ptr(), 8192, 4, 16, 2, sink.data_ptr(), None) == 0
+        torch.cuda.synchronize()
+        pairs = int(sink[2:4].view(torch.int64).item())
+        cells = 4 * 2 * 2048                                    # CTAs x work items x queries
+        assert 5.0 < pairs / cells < 6.5                        # the mean of Binomial(46, 1/8) is 5.75
+    assert lib.psattn_probe_gather(13, rows.data_ptr(), 1024, 4, 16, 2, sink.data_ptr(), None) == 2     # buffer too small
+    assert lib.psattn_probe_gather(13, rows.data_ptr(), 8192, 4, 8, 2, sink.data_ptr(), None) == 2      # 16 warps only
+
+
 def test_bad_arguments_are_refused():
     lib = ps.load()
     sink = torch.zeros(4, dtype=torch.int32, device="cuda")

@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(768, 1) k_probe_bulk(const uint4 *__restrict__
 // Binomial(U, 1/8) samples in one of eight chunks; the mma layout gives each of a warp's eight queries two rows per
 // round, so a group of eight costs max over its queries of ceil(n / 2) rounds.  Per work item (one chunk, 2048
 // queries): the chunk is copied in, then every warp takes groups of eight queries - their rows of Q staged through
-// shared memory (cp.async, one group ahead) and read as mma fragments, their row numbers read from a table, the rounds
+// shared memory (cp.async, three groups ahead) and read as mma fragments, their row numbers read from a table, the rounds
 // as in k_probe_smem_mma.  kSorted: the counts of a group are neighbours in the sorted order of their 128-query block
 // (what a pre-pass that orders the queries of a block by count would deliver); otherwise they are independent draws.
 // counts: 128 quantiles of the count distribution.  The kernel adds the useful pairs to sink[2..3] (64 bit).
@@ -276,8 +276,9 @@ __global__ void __launch_bounds__(512, 1) k_probe_bucketed(const uint4 *__restri
                                                            ProbeCounts counts, uint32_t *__restrict__ sink) {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr int kQueries = 2048;
-    uint8_t *qstage = smem + kProbeSmemRows * 128;                       // [16 warps][2][1 KB]
-    uint32_t *table = reinterpret_cast<uint32_t *>(qstage + 16 * 2 * 1024);   // 4096 row numbers
+    constexpr int kAhead = 3;                                            // groups of Q rows requested ahead of the one in work
+    uint8_t *qstage = smem + kProbeSmemRows * 128;                       // [16 warps][kAhead + 1][1 KB]
+    uint32_t *table = reinterpret_cast<uint32_t *>(qstage + 16 * (kAhead + 1) * 1024);   // 4096 row numbers
     unsigned char *cnt = reinterpret_cast<unsigned char *>(table + 4096);     // counts of the item's queries
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int e = tid; e < 4096; e += blockDim.x) table[e] = probe_hash((uint32_t)e * 7919u + blockIdx.x) % kProbeSmemRows;
@@ -299,7 +300,7 @@ __global__ void __launch_bounds__(512, 1) k_probe_bucketed(const uint4 *__restri
             cnt[q] = kSorted ? counts.q[q & 127] : counts.q[probe_hash(work * 4096u + (uint32_t)q) & 127];
         __syncthreads();
         const uint32_t q0 = (work * 2048u + 12345u) % (n_rows - 2048u);  // the item's rows of Q, consecutive
-        uint8_t *st = qstage + warp * 2048;
+        uint8_t *st = qstage + warp * (kAhead + 1) * 1024;
         auto stage_q = [&](int grp, int buf) {                           // 8 rows x 128 B: two 16-byte pieces per lane
             const uint4 *src = rows + (size_t)(q0 + grp * 8) * 8;
 #pragma unroll
@@ -311,13 +312,15 @@ __global__ void __launch_bounds__(512, 1) k_probe_bucketed(const uint4 *__restri
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
         int it = 0;
-        stage_q(warp, 0);
+        for (int a = 0; a < kAhead; ++a) stage_q(warp + 16 * a, a);      // (2048 queries: every warp has 16 groups)
         for (int grp = warp; grp < kQueries / 8; grp += 16, ++it) {
-            if (grp + 16 < kQueries / 8) { stage_q(grp + 16, (it + 1) & 1); asm volatile("cp.async.wait_group 1;" ::: "memory"); }
-            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            // one commit per trip, empty at the end, so that "all but the newest kAhead groups" is always this trip's rows
+            if (grp + 16 * kAhead < kQueries / 8) stage_q(grp + 16 * kAhead, (it + kAhead) % (kAhead + 1));
+            else asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group %0;" ::"n"(kAhead) : "memory");
             __syncwarp();
             uint32_t bq[8];
-            const uint32_t qa = sm100::smem_u32(st + (it & 1) * 1024) + (uint32_t)l7 * 128u;
+            const uint32_t qa = sm100::smem_u32(st + (it % (kAhead + 1)) * 1024) + (uint32_t)l7 * 128u;
             asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                          : "=r"(bq[0]), "=r"(bq[1]), "=r"(bq[2]), "=r"(bq[3]) : "r"(qa + (uint32_t)((((lane >> 3) + l7) & 7) << 4)));
             asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -457,7 +460,7 @@ extern "C" int psattn_probe_gather(int32_t mode, const void *rows, int64_t n_row
                 pc.q[i] = (unsigned char)k;
             }
         }
-        const size_t smem = (size_t)kProbeSmemRows * 128 + 16 * 2 * 1024 + 4096 * 4 + 2048;
+        const size_t smem = (size_t)kProbeSmemRows * 128 + 16 * 4 * 1024 + 4096 * 4 + 2048;
         static SmemGrant g13, g14;
         const dim3 grid((unsigned)n_ctas), block(512);
         if (mode == 13) {

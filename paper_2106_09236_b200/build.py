@@ -31,11 +31,15 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, phase_stamps: bool = False) -> str:
-    """Builds the library.  phase_stamps: a second library, libpsattn_stamps.so, whose fused forward kernel
-    accumulates per-phase times (-DPSATTN_PHASE_STAMPS); only the benchmark's --phases mode uses it."""
+def build(force: bool = False, verbose: bool = False, phase_stamps: bool = False, nvtx: bool = False) -> str:
+    """Builds the library.  phase_stamps: a second library, libpsattn_stamps.so, whose kernels record per-phase
+    times and their begin and end (-DPSATTN_PHASE_STAMPS); only the benchmark's --phases mode uses it.
+    nvtx: a library, libpsattn_nvtx.so, with a named range around every compute entry point (-DPSATTN_NVTX) for
+    timeline tools; load it with PSATTN_LIBRARY."""
     if phase_stamps:
         return _build_variant("libpsattn_stamps.so", ["-DPSATTN_PHASE_STAMPS"], ".stamps.o")
+    if nvtx:
+        return _build_variant("libpsattn_nvtx.so", ["-DPSATTN_NVTX"], ".nvtx.o", ["-ldl"])
     if not force and not needs_build():
         return LIB
     objs = []
@@ -54,7 +58,7 @@ def build(force: bool = False, verbose: bool = False, phase_stamps: bool = False
     return LIB
 
 
-def _build_variant(name: str, extra: list, suffix: str) -> str:
+def _build_variant(name: str, extra: list, suffix: str, link: list = ()) -> str:
     out = os.path.join(HERE, name)
     objs = []
     for src in SOURCES:
@@ -62,10 +66,10 @@ def _build_variant(name: str, extra: list, suffix: str) -> str:
         subprocess.check_call([_nvcc(), *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj])
         objs.append(obj)
     tmp = out + ".tmp.%d" % os.getpid()
-    subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart"])
+    subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-lcudart", *link])
     os.replace(tmp, out)
     return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, nvtx="--nvtx" in sys.argv))

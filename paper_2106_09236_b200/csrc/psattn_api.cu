@@ -38,6 +38,21 @@ struct psattn_plan {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Named ranges around the compute entry points for timeline tools, compiled in only with -DPSATTN_NVTX (a separate
+// build of the library; the regular one contains no call into the tools interface).
+#ifdef PSATTN_NVTX
+#include <nvtx3/nvToolsExt.h>
+struct ApiRange {
+    explicit ApiRange(const char *name) { nvtxRangePushA(name); }
+    ~ApiRange() { nvtxRangePop(); }
+};
+#else
+struct ApiRange {
+    explicit ApiRange(const char *) {}
+};
+#endif
+#define PSATTN_RANGE() ApiRange api_range_(__func__)
+
 extern "C" int psattn_version(void) { return 1000; }
 
 extern "C" const char *psattn_status_string(int s) {
@@ -381,6 +396,7 @@ extern "C" int psattn_forward(psattn_plan_t *plan, const void *Q, const void *K,
                               const int32_t *lengths, const int32_t *sample_idx, void *O,
                               int32_t *sel_idx, float *M_out, void *workspace,
                               size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !V || !sample_idx || !O || !sel_idx) return PSATTN_ERR_NULL;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return PSATTN_ERR_MISALIGNED;
     int rc = check_ws(plan, workspace, workspace_bytes);
@@ -435,6 +451,7 @@ extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q,
                                              const void *V, const int32_t *lengths,
                                              const int32_t *sel_idx_in, void *O, void *workspace,
                                              size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !V || !sel_idx_in || !O) return PSATTN_ERR_NULL;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return PSATTN_ERR_MISALIGNED;
     int rc = check_ws(plan, workspace, workspace_bytes);
@@ -461,6 +478,7 @@ extern "C" int psattn_forward_with_selection(psattn_plan_t *plan, const void *Q,
 extern "C" int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K,
                               const int32_t *lengths, const int32_t *sample_idx, float *M_out,
                               void *workspace, size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !sample_idx || !M_out) return PSATTN_ERR_NULL;
     if (!aligned16(Q) || !aligned16(K)) return PSATTN_ERR_MISALIGNED;
     int rc = check_ws(plan, workspace, workspace_bytes);
@@ -471,6 +489,7 @@ extern "C" int psattn_measure(psattn_plan_t *plan, const void *Q, const void *K,
 
 extern "C" int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const void *K, const int32_t *lengths,
                                     float *M_out, void *workspace, size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !M_out) return PSATTN_ERR_NULL;
     if (!aligned16(Q) || !aligned16(K)) return PSATTN_ERR_MISALIGNED;
     int rc = check_ws(plan, workspace, workspace_bytes);
@@ -486,6 +505,7 @@ extern "C" int psattn_exact_measure(psattn_plan_t *plan, const void *Q, const vo
 extern "C" int psattn_project_qkv(psattn_plan_t *plan, const void *X, const void *Wt, int32_t d_x,
                                   const int32_t *lengths, void *Q, void *K, void *V, float *vbar,
                                   void *workspace, size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !X || !Wt || !Q || !K || !V) return PSATTN_ERR_NULL;
     if (d_x < 1 || d_x > (1 << 20)) return PSATTN_ERR_BAD_DESC;
     if (!aligned16(X) || !aligned16(Wt) || !aligned16(Q) || !aligned16(K) || !aligned16(V)) return PSATTN_ERR_MISALIGNED;
@@ -501,6 +521,7 @@ extern "C" int psattn_project_qkv(psattn_plan_t *plan, const void *X, const void
 extern "C" int psattn_project_out(psattn_plan_t *plan, const void *O, const int32_t *sel_idx, const int32_t *lengths,
                                   const void *Wot, int32_t d_y, void *Y, void *workspace, size_t workspace_bytes,
                                   void *stream) {
+    PSATTN_RANGE();
     if (!plan || !O || !Wot || !Y) return PSATTN_ERR_NULL;
     if (d_y < 1 || d_y > (1 << 20)) return PSATTN_ERR_BAD_DESC;
     if (!aligned16(O) || !aligned16(Wot) || !aligned16(Y)) return PSATTN_ERR_MISALIGNED;
@@ -519,6 +540,7 @@ extern "C" int psattn_project_out(psattn_plan_t *plan, const void *O, const int3
 extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t *lengths,
                              int32_t *sel_idx, void *workspace, size_t workspace_bytes,
                              void *stream) {
+    PSATTN_RANGE();
     if (!plan || !M || !sel_idx) return PSATTN_ERR_NULL;
     int rc = check_ws(plan, workspace, workspace_bytes);
     if (rc) return rc;
@@ -530,6 +552,7 @@ extern "C" int psattn_select(psattn_plan_t *plan, const float *M, const int32_t 
 
 extern "C" int psattn_mean_v(psattn_plan_t *plan, const void *V, const int32_t *lengths,
                              float *vbar, void *workspace, size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !V || !vbar) return PSATTN_ERR_NULL;
     if (!aligned16(V)) return PSATTN_ERR_MISALIGNED;
     int rc = check_ws(plan, workspace, workspace_bytes);
@@ -545,6 +568,7 @@ extern "C" int psattn_attend_rows(psattn_plan_t *plan, const void *Q, const void
                                   const int32_t *lengths, const int32_t *row_idx, int32_t n_rows,
                                   float *out, void *workspace, size_t workspace_bytes,
                                   void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !V || !row_idx || !out) return PSATTN_ERR_NULL;
     if (n_rows < 0 || n_rows > plan->u_max) return PSATTN_ERR_BAD_DESC;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V)) return PSATTN_ERR_MISALIGNED;
@@ -559,6 +583,7 @@ extern "C" int psattn_attend_rows(psattn_plan_t *plan, const void *Q, const void
 extern "C" int psattn_dense_forward(psattn_plan_t *plan, const void *Q, const void *K,
                                     const void *V, const int32_t *lengths, void *O,
                                     void *workspace, size_t workspace_bytes, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !V || !O) return PSATTN_ERR_NULL;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return PSATTN_ERR_MISALIGNED;
     int rc = check_ws(plan, workspace, workspace_bytes);
@@ -614,6 +639,7 @@ extern "C" int psattn_plan_enable_host_io(psattn_plan_t *plan) {
 extern "C" int psattn_forward_host(psattn_plan_t *plan, const void *Q, const void *K, const void *V,
                                    const int32_t *lengths, const int32_t *sample_idx, void *O,
                                    int32_t *sel_idx, void *stream) {
+    PSATTN_RANGE();
     if (!plan || !Q || !K || !V || !sample_idx || !O || !sel_idx) return PSATTN_ERR_NULL;
     if (!plan->host_io) return PSATTN_ERR_BAD_DESC;
     if (int rc = check_device(plan)) return rc;

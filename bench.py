@@ -66,12 +66,12 @@ _FUSED_SOURCES = ["psattn_fused.cu", "psattn_measure_mma.cuh", "psattn_attend64.
 _STREAM_SOURCES = ["psattn_measure_mma.cu", "psattn_measure_stream.cuh", "psattn_measure_mma.cuh",
                    "psattn_sm100.cuh", "psattn_common.cuh"]
 TRAFFIC = {
-    "large_bf16": {"kernel": "k_forward_fused", "bytes": 53289216, "sources": _FUSED_SOURCES,
+    "large_bf16": {"kernel": "k_forward_fused", "bytes": 54344192, "sources": _FUSED_SOURCES,
                    "profile": "profiles/ncu_full_k_forward_fused_large_bf16.txt",
-                   "sources_sha1": "f3ff2aa00e21e35a01acf6d8a3cdd80d10ab35e8"},
-    "long_bf16": {"kernel": "k_measure_stream", "bytes": 76287488, "sources": _STREAM_SOURCES,
+                   "sources_sha1": "605a5cec63dc810331d622f1397e716836f31c53"},
+    "long_bf16": {"kernel": "k_measure_stream", "bytes": 75986944, "sources": _STREAM_SOURCES,
                   "profile": "profiles/ncu_full_k_measure_stream_long_bf16.txt",
-                  "sources_sha1": "43d7f08d36d6498c4d5d9217d174735396085acf"},
+                  "sources_sha1": "3d85716f75af55982a00d06ed97d69c0403d17ba"},
 }
 
 

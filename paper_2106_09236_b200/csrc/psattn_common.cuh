@@ -155,6 +155,7 @@ __device__ __forceinline__ MeasureState measure_merge(const MeasureState &a, con
 // Order-preserving map float -> uint32 (larger float <=> larger key).
 __device__ __forceinline__ unsigned float_key(float f) {
     unsigned b = __float_as_uint(f);
+    if (b == 0x80000000u) b = 0u;                          // -0 and +0 are one value: they tie, the lower position first
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 

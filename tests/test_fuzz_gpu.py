@@ -3,11 +3,12 @@ kernels' regimes (tile sizes, the longest sequence the fused kernel takes), ragg
 schedules, both fills, the count rules of Sec. 3.2."""
 import numpy as np
 import pytest
+import torch
 
 import parity
 from oracle import psattn_oracle as orc
 from paper_2106_09236_b200 import binding as ps
-from test_parity_gpu import _run_forward, _synth
+from test_parity_gpu import _dev, _run_forward, _synth
 
 pytestmark = pytest.mark.gpu
 
@@ -65,3 +66,55 @@ def test_random_shapes_match_the_oracle(seed):
             parity.check_forward(O, sel, M, inp, inp["lengths"], k["dtype"], k["c"], **k["check_kw"])
         except AssertionError as e:
             raise AssertionError("case %r: %s" % ({x: k[x] for x in k if x != "check_kw"}, e))
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_dense_row_list_and_selection_calls_match_the_oracle(seed):
+    """The per-step entry points on random shapes: the dense comparator, step (d) for random row lists (few rows:
+    the 64-row kernel; with a larger u: the 256-row kernel; holes and repeated rows included) and step (c) on
+    random values with heavy ties and zeros of both signs."""
+    rng = np.random.default_rng(seed)
+    for it in range(30):
+        T = int(rng.choice([rng.integers(1, 300), rng.choice([127, 128, 129, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025]),
+                            rng.integers(300, 2600)]))
+        B, H = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        dtype = "bf16" if rng.random() < 0.8 else "fp32"
+        lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+        inp = _synth(B, H, T, 7000 + it, 4, dtype, lengths)
+        dev, tdt = _dev(inp, dtype)
+        u_over = int(rng.integers(65, 300)) if (dtype == "bf16" and T > 300 and rng.random() < 0.4) else 0
+        plan = ps.Plan(B, H, T, dtype=tdt, c=5.0, u_override=u_over)
+        what = dict(B=B, H=H, T=T, dtype=dtype, lengths=lengths, u_override=u_over)
+        if T <= 1300:
+            O = plan.psattn_dense_forward(dev["Q"], dev["K"], dev["V"], dev["lengths"])
+            torch.cuda.synchronize()
+            ref = orc.dense(inp["Q"], inp["K"], inp["V"], inp["lengths"], nthreads=8)
+            assert np.abs(O.float().cpu().numpy() - ref).max() <= parity.O_ATOL[dtype], what
+        n_rows = int(rng.integers(1, plan.u_max + 1))
+        rows = np.stack([[rng.integers(0, lengths[b], size=n_rows) for _ in range(H)] for b in range(B)]).astype(np.int32)
+        rows[rng.random(rows.shape) < 0.05] = -1
+        if T > 3:
+            rows[0, 0, 0] = T - 1
+        out = plan.psattn_attend_rows(dev["Q"], dev["K"], dev["V"], dev["lengths"], torch.from_numpy(rows).cuda())
+        torch.cuda.synchronize()
+        out = out.cpu().numpy()
+        # fp32 rows out; with bf16 inputs the weights are rounded to bf16 (2^-9 relative) before they meet |V| <= 4
+        tol = 1e-4 if dtype == "fp32" else 8e-3
+        for b in range(B):
+            for h in range(H):
+                for r in rng.choice(n_rows, size=min(n_rows, 6), replace=False):
+                    i = int(rows[b, h, r])
+                    if i < 0 or i >= lengths[b]:
+                        assert np.all(out[b, h, r] == 0.0), what
+                    else:
+                        ref = orc.attend_row(inp["Q"], inp["K"], inp["V"], b, h, i, lengths[b])
+                        assert np.abs(out[b, h, r] - ref).max() <= tol, what
+        M = rng.standard_normal((B, H, T)).astype(np.float32)
+        if rng.random() < 0.5:
+            M = np.round(M * 2) / 2                           # steps of 0.5: many ties, -0.0 and +0.0 among them
+        sel = plan.psattn_select(torch.from_numpy(M).cuda(), dev["lengths"])
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(sel.cpu().numpy(), orc.select(M.astype(np.float64), np.asarray(lengths, dtype=np.int32),
+                                                                    c=5.0, u_override=u_over, u_max=plan.u_max), err_msg=repr(what))
+        assert plan.psattn_read_status() == 0, what
+        plan.close()

@@ -356,6 +356,23 @@ def test_zero_queries_pick_lowest_indices_and_output_mean():
             np.testing.assert_allclose(O[b, h, :L], np.broadcast_to(vb[b, h], (L, d)), atol=1e-13)
 
 
+# ---- signed zeros are one value -------------------------------------------------------------
+
+def test_signed_zeros_tie_in_the_selection():
+    """-0.0 and +0.0 compare equal, so among them the lower position wins (the tie rule), whatever their signs;
+    checked against a stable sort of the values."""
+    T, c = 40, 5.0
+    rng = np.random.default_rng(77)
+    M = np.where(rng.random((1, 1, T)) < 0.5, 0.0, -0.0)
+    M[0, 0, [5, 17, 30]] = [1.0, -1.0, 2.0]
+    u = brute.n_count(c, T)
+    order = np.argsort(-M[0, 0], kind="stable")             # equal values keep their position order
+    want = np.sort(order[:u])
+    sel = orc.select(M, np.array([T], dtype=np.int32), c=c)
+    assert [int(x) for x in sel[0, 0] if x >= 0] == [int(x) for x in want]
+    assert 17 not in want and 5 in want and 30 in want
+
+
 # ---- P11: planted spikes ---------------------------------------------------------------
 
 def test_planted_spikes_are_selected():

@@ -464,6 +464,22 @@ def test_select_entry_point_is_exact_including_ties():
     plan.close()
 
 
+@pytest.mark.parametrize("T", [40, 700, 2500])
+def test_select_treats_signed_zeros_as_one_value(T):
+    """-0.0 and +0.0 are equal values: they tie, the lower position first, as in the oracle."""
+    B, H, c = 2, 2, 5.0
+    rng = np.random.default_rng(70 + T)
+    M = np.where(rng.random((B, H, T)) < 0.5, 0.0, -0.0).astype(np.float32)
+    M[0, 0, ::11] = rng.standard_normal(M[0, 0, ::11].shape).astype(np.float32)     # a few real values of both signs
+    M[1, 1] = np.round(rng.standard_normal(T) * 2) / 2                              # steps of 0.5: zeros of both signs among them
+    lengths = np.array([T, max(1, T - 13)], dtype=np.int32)
+    plan = ps.Plan(B, H, T, c=c)
+    sel = plan.psattn_select(torch.from_numpy(M).cuda(), torch.from_numpy(lengths).cuda())
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(sel.cpu().numpy(), orc.select(M.astype(np.float64), lengths, c=c, u_max=plan.u_max))
+    plan.close()
+
+
 @pytest.mark.parametrize("B,H,T", [(3, 2, 9000), (4, 8, 8192), (1, 1, 8200)])
 def test_select_of_few_long_units_is_exact_including_ties(B, H, T):
     """Few units of long sequences are selected range by range and then among the ranges' candidates:

@@ -8,7 +8,7 @@ import torch
 import parity
 from oracle import psattn_oracle as orc
 from paper_2106_09236_b200 import binding as ps
-from test_parity_gpu import _dev, _run_forward, _synth
+from test_parity_gpu import _dev, _run_forward, _shared_sample, _synth
 
 pytestmark = pytest.mark.gpu
 
@@ -118,3 +118,90 @@ def test_random_dense_row_list_and_selection_calls_match_the_oracle(seed):
                                                                     c=5.0, u_override=u_over, u_max=plan.u_max), err_msg=repr(what))
         assert plan.psattn_read_status() == 0, what
         plan.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_index_layouts_strides_and_reused_selections_match_the_oracle(seed):
+    """Per-head sample arrays, one sample per sequence, U overrides, the [B][T][H][d] layout through the stride fields,
+    and a selection computed on one set of tensors reused on another (Sec. 4.4), on random shapes."""
+    rng = np.random.default_rng(seed)
+    c, d = 5.0, 64
+    for it in range(24):
+        T = int(rng.choice([rng.integers(2, 300), rng.choice([255, 256, 257, 1023, 1024, 1025, 1099, 1100, 1101]),
+                            rng.integers(300, 2600)]))
+        B, H = int(rng.integers(1, 4)), int(rng.integers(1, 5))
+        dtype = "bf16" if rng.random() < 0.75 else "fp32"
+        lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+        path = [ps.PSATTN_PATH_AUTO, ps.PSATTN_PATH_STAGED][int(rng.integers(0, 2))]
+        U_over = int(rng.choice([0, 0, rng.integers(1, 64)]))
+        n_cols = max(max(orc.count(c, L) for L in range(1, T + 1)), U_over)
+        inp = _synth(B, H, T, 5000 + it, n_cols, dtype, lengths)
+        mode = int(rng.integers(0, 4))
+        what = dict(B=B, H=H, T=T, dtype=dtype, lengths=lengths, path=path, U_override=U_over, mode=mode)
+        if mode == 0:
+            idx = rng.integers(0, np.asarray(lengths)[:, None, None, None], size=(B, H, T, n_cols)).astype(np.int32)
+            O, sel, M, status = _run_forward(dict(inp, sample_idx=idx), dtype, c, path, idx_per_head=True, U_override=U_over)
+            assert status == 0, what
+            parity.check_forward(O, sel, M, dict(inp, sample_idx=idx), inp["lengths"], dtype, c, U_override=U_over)
+        elif mode == 1:
+            compact, expanded = _shared_sample(inp)
+            O, sel, M, status = _run_forward(dict(inp, sample_idx=compact), dtype, c, path, idx_shared=True, U_override=U_over)
+            assert status == 0, what
+            parity.check_forward(O, sel, M, dict(inp, sample_idx=expanded), inp["lengths"], dtype, c, U_override=U_over)
+        elif mode == 2:
+            dev, tdt = _dev(inp, dtype)
+            st = (T * H * d, d, H * d)
+            perm = {k: dev[k].permute(0, 2, 1, 3).contiguous() for k in ("Q", "K", "V")}
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n_cols, path=path, U_override=U_over,
+                           strides={"q": st, "k": st, "v": st, "o": st})
+            O = torch.full((B, T, H, d), float("nan"), dtype=tdt, device="cuda")
+            sel = torch.empty((B, H, plan.u_max), dtype=torch.int32, device="cuda")
+            M = torch.empty((B, H, T), dtype=torch.float32, device="cuda")
+            plan.psattn_forward(perm["Q"], perm["K"], perm["V"], dev["lengths"], dev["sample_idx"], O, sel, M)
+            torch.cuda.synchronize()
+            assert plan.psattn_read_status() == 0, what
+            parity.check_forward(O.permute(0, 2, 1, 3).float().cpu().numpy(), sel.cpu().numpy(), M.cpu().numpy(), inp,
+                                 inp["lengths"], dtype, c, U_override=U_over)
+            plan.close()
+        else:
+            dev, tdt = _dev(inp, dtype)
+            inp2 = _synth(B, H, T, 6000 + it, n_cols, dtype, lengths)
+            dev2, _ = _dev(inp2, dtype)
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n_cols, path=path, U_override=U_over)
+            _, sel = plan.psattn_forward(dev["Q"], dev["K"], dev["V"], dev["lengths"], dev["sample_idx"])
+            O2 = plan.psattn_forward_with_selection(dev2["Q"], dev2["K"], dev2["V"], dev["lengths"], sel)
+            torch.cuda.synchronize()
+            assert plan.psattn_read_status() == 0, what
+            O2, s_host = O2.float().cpu().numpy(), sel.cpu().numpy()
+            vbar = orc.mean_v(inp2["V"], inp["lengths"])
+            for b in range(B):
+                L = lengths[b]
+                for h in range(H):
+                    chosen = set(int(x) for x in s_host[b, h] if x >= 0)
+                    for i in list(chosen)[:4] + [int(x) for x in rng.integers(0, L, size=4)]:
+                        ref = orc.attend_row(inp2["Q"], inp2["K"], inp2["V"], b, h, i, L) if i in chosen else vbar[b, h]
+                        assert np.abs(O2[b, h, i] - ref).max() <= parity.O_ATOL[dtype], what
+                    assert np.all(O2[b, h, L:] == 0.0), what
+            plan.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_projection_shapes_match_the_oracle(seed):
+    """The projections in front of the path on random widths (multiples of 64, of 8, and widths the tensor map cannot
+    take), head counts, lengths with empty sequences, NaN in the padding."""
+    import test_projection_gpu as tpj
+    from paper_2106_09236_b200 import workloads as wl
+    rng = np.random.default_rng(seed)
+    for it in range(20):
+        B, H = int(rng.integers(1, 4)), int(rng.integers(1, 7))
+        T = int(rng.choice([rng.integers(1, 200), rng.choice([127, 128, 129, 255, 256, 257, 383, 384, 385]), rng.integers(200, 900)]))
+        dx = int(rng.choice([8 * rng.integers(1, 80), 64 * rng.integers(1, 9), 512, 4 * rng.integers(1, 30) + 2]))
+        lengths = [int(rng.integers(0, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+        X = wl.round_to_bf16(rng.standard_normal((B, T, dx), dtype=np.float32))
+        Wt = wl.round_to_bf16(rng.standard_normal((3, H * 64, dx), dtype=np.float32) / np.float32(np.sqrt(dx)))
+        inp = {"X": X, "Wt": Wt, "lengths": np.array(lengths, dtype=np.int32)}
+        for b, L in enumerate(lengths):
+            inp["X"][b, L:] = np.nan                              # never read
+        res, vbar = tpj._run(inp, H, "bf16")
+        inp["X"] = np.nan_to_num(inp["X"], nan=0.0)
+        tpj._compare(inp, H, "bf16", res, vbar)

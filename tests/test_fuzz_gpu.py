@@ -205,3 +205,33 @@ def test_random_projection_shapes_match_the_oracle(seed):
         res, vbar = tpj._run(inp, H, "bf16")
         inp["X"] = np.nan_to_num(inp["X"], nan=0.0)
         tpj._compare(inp, H, "bf16", res, vbar)
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_counts_around_64_long_ragged_and_many_short_units(seed):
+    """c chosen so that u and U fall around 63 / 64 / 65 (the limits of the 64-row attention kernel, of the fused
+    kernel and of the tensor-datapath measure kernels), sequences of 3000-10000 positions with ragged lengths, and
+    batches of many short units."""
+    rng = np.random.default_rng(seed)
+    for it in range(18):
+        kind = int(rng.integers(0, 3))
+        if kind == 0:
+            T = int(rng.choice([rng.integers(900, 1101), rng.integers(1101, 3000)]))
+            c, B, H = float(rng.uniform(8.4, 9.8)), int(rng.integers(1, 3)), int(rng.integers(1, 4))
+        elif kind == 1:
+            T, c, B, H = int(rng.integers(3000, 10000)), 5.0, int(rng.integers(1, 4)), int(rng.integers(1, 9))
+        else:
+            T, c = int(rng.integers(1, 200)), float(rng.choice([1.0, 5.0, 12.0]))
+            B, H = int(rng.integers(4, 40)), int(rng.integers(1, 9))
+        dtype = "bf16" if rng.random() < 0.85 else "fp32"
+        lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.7 else T for _ in range(B)]
+        path = [ps.PSATTN_PATH_AUTO, ps.PSATTN_PATH_STAGED][int(rng.integers(0, 2))]
+        n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+        inp = _synth(B, H, T, 3000 + it, n_cols, dtype, lengths)
+        what = dict(B=B, H=H, T=T, c=c, dtype=dtype, lengths=lengths[:6], path=path, U=n_cols)
+        O, sel, M, status = _run_forward(inp, dtype, c, path)
+        assert status == 0, what
+        try:
+            parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c)
+        except AssertionError as e:
+            raise AssertionError("case %r: %s" % (what, e))

@@ -36,6 +36,7 @@ struct OutArgs {
 };
 
 __host__ __device__ inline uint32_t po_w_pitch(int H) { return (uint32_t)(H * 64 + 8) * 2u; }   // bytes per weight row
+__host__ __device__ inline size_t po_align16(size_t x) { return (x + 15) / 16 * 16; }
 
 __device__ __forceinline__ void po_mma(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                        uint32_t b1) {
@@ -60,8 +61,11 @@ __global__ void __launch_bounds__(kPoThreads, 1) k_project_out_rows(OutArgs a) {
     int *pair_t = reinterpret_cast<int *>(base + 64);                                       // [max_pairs] position, -1 = padding
     int *slot_t = pair_t + a.max_pairs;                                                     // [max_slots] position of a slot
     short *pair_of = reinterpret_cast<short *>(slot_t + a.max_slots);                       // [H][max_slots] pair of (head, slot) or -1
-    short *slot_of = pair_of + (size_t)a.H * a.max_slots;                                   // [t_chunk] slot of a position or -1
-    float *P = reinterpret_cast<float *>(reinterpret_cast<uint8_t *>(slot_of) + ((a.t_chunk * 2 + 15) / 16) * 16);   // [max_pairs][64]
+    // (H * max_slots may be odd: the arrays behind it start on the next 16-byte boundary of the block's memory)
+    short *slot_of = reinterpret_cast<short *>(smem + po_align16((size_t)(reinterpret_cast<uint8_t *>(pair_of) - smem) +
+                                                                 (size_t)a.H * a.max_slots * 2));   // [t_chunk] slot of a position or -1
+    float *P = reinterpret_cast<float *>(smem + po_align16((size_t)(reinterpret_cast<uint8_t *>(slot_of) - smem) +
+                                                           (size_t)a.t_chunk * 2));              // [max_pairs][64]
 
     pdl_enter();
     int L = a.lengths ? a.lengths[b] : a.T;
@@ -337,9 +341,12 @@ cudaError_t launch_project_out(int dtype, int mode, const Geom &g, int dy, const
         a.t_chunk = t_chunk;
         a.max_slots = g.H * g.u_max < t_chunk ? g.H * g.u_max : t_chunk;
         a.max_pairs = g.H * ((g.u_max + 15) / 16 * 16);         // every head's rows padded to whole 16-row tiles
-        const size_t smem = (size_t)kPoCols * po_w_pitch(g.H) + (size_t)g.H * 64 * 2 +
-                            (size_t)g.H * 64 * 4 + 64 * 4 + (size_t)a.max_pairs * 4 + (size_t)a.max_slots * 4 + (size_t)g.H * a.max_slots * 2 +
-                            ((size_t)t_chunk * 2 + 15) / 16 * 16 + (size_t)a.max_pairs * 64 * 4 + 128;
+        // the kernel's layout: weights, fill rows, c, base, pair positions, slot positions, pair_of | slot_of | P
+        size_t smem = (size_t)kPoCols * po_w_pitch(g.H) + (size_t)g.H * 64 * 2 + (size_t)g.H * 64 * 4 + 64 * 4 +
+                      (size_t)a.max_pairs * 4 + (size_t)a.max_slots * 4;
+        smem = po_align16(smem + (size_t)g.H * a.max_slots * 2);
+        smem = po_align16(smem + (size_t)t_chunk * 2);
+        smem += (size_t)a.max_pairs * 64 * 4 + 128;
         if (smem <= 200 * 1024 && chunks <= 65535 && g.B <= 65535) {
             static SmemGrant grant;
             if (cudaError_t e = grant_dynamic_smem(k_project_out_rows, grant, smem)) return e;

@@ -235,3 +235,26 @@ def test_random_counts_around_64_long_ragged_and_many_short_units(seed):
             parity.check_forward(O, sel, M, inp, inp["lengths"], dtype, c)
         except AssertionError as e:
             raise AssertionError("case %r: %s" % (what, e))
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_output_matrix_shapes_match_the_oracle(seed):
+    """The output matrix behind the path, both forms, on random head counts (odd ones included), widths, lengths."""
+    import test_project_out_gpu as tpo
+    from paper_2106_09236_b200 import workloads as wl
+    rng = np.random.default_rng(seed)
+    for it in range(20):
+        H, B = int(rng.integers(1, 9)), int(rng.integers(1, 5))
+        T = int(rng.choice([rng.integers(1, 300), rng.choice([127, 128, 129, 255, 256, 257]), rng.integers(300, 2200)]))
+        c = float(rng.choice([5.0, 5.0, 2.0, 9.0]))
+        dy = int(rng.choice([64 * rng.integers(1, 9), 8 * rng.integers(1, 70), 512]))
+        lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+        n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+        if n_cols > 64:
+            c = 5.0
+            n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+        wk = wl.Workload("adhoc", 0, B, H, T, 64, "bf16", c, 0.1, 3.0)
+        inp = wl.make_inputs(wk, n_cols, seed=8000 + it, lengths=lengths)
+        plan, O, sel, lens, tdt = tpo._forward(inp, "bf16", c)
+        tpo._run_all_forms(plan, O, sel, lens, tpo._weights(H, dy, 9 + it, "bf16"), tdt, "bf16", inp["lengths"])
+        plan.close()

@@ -86,6 +86,20 @@ def test_output_matrix_odd_widths_short_sequences_and_full_selection(dy):
     plan.close()
 
 
+@pytest.mark.parametrize("H,T", [(1, 1322), (7, 1086), (3, 175), (5, 64)])
+def test_output_matrix_with_odd_head_counts(H, T):
+    """H times the number of slots odd: the arrays behind the (head, slot) table of the shortcut kernel must still
+    start on 16-byte boundaries of its shared memory."""
+    c = 5.0
+    lengths = [T, max(1, T // 2), max(1, T - 5)]
+    n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+    wk = wl.Workload("adhoc", 0, len(lengths), H, T, 64, "bf16", c, 0.1, 3.0)
+    inp = wl.make_inputs(wk, n_cols, seed=64 + H, lengths=lengths)
+    plan, O, sel, lens, tdt = _forward(inp, "bf16", c)
+    _run_all_forms(plan, O, sel, lens, _weights(H, 256, 8, "bf16"), tdt, "bf16", inp["lengths"])
+    plan.close()
+
+
 def test_output_matrix_with_a_given_selection_shared_by_all_heads():
     """Every head selects the same positions (the most corrections a row can collect), through
     psattn_forward_with_selection."""

@@ -258,3 +258,89 @@ def test_random_output_matrix_shapes_match_the_oracle(seed):
         plan, O, sel, lens, tdt = tpo._forward(inp, "bf16", c)
         tpo._run_all_forms(plan, O, sel, lens, tpo._weights(H, dy, 9 + it, "bf16"), tdt, "bf16", inp["lengths"])
         plan.close()
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_calls_of_the_other_entry_points_match_the_oracle(seed):
+    """The exact measure of Eq. 10, mean(V), the sampled measure alone on long ragged sequences, row lists over long sequences (key splits and their merge), and the
+    host-buffer front end."""
+    rng = np.random.default_rng(seed)
+    for it in range(20):
+        mode = int(rng.integers(0, 5))
+        B, H = int(rng.integers(1, 4)), int(rng.integers(1, 6))
+        dtype = "bf16" if rng.random() < 0.75 else "fp32"
+        path = [ps.PSATTN_PATH_AUTO, ps.PSATTN_PATH_STAGED][int(rng.integers(0, 2))]
+        c = 5.0
+        what = dict(mode=mode, B=B, H=H, dtype=dtype, path=path)
+        if mode == 0:      # exact measure
+            T = int(rng.choice([rng.integers(1, 200), rng.choice([127, 128, 129, 255, 256, 257, 511, 512, 513]), rng.integers(200, 900)]))
+            lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+            what.update(T=T, lengths=lengths)
+            inp = _synth(B, H, T, 100 + it, orc.count(c, T), dtype, lengths)
+            dev, tdt = _dev(inp, dtype)
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c, path=path)
+            M = plan.psattn_exact_measure(dev["Q"], dev["K"], dev["lengths"]); torch.cuda.synchronize()
+            assert plan.psattn_read_status() == 0
+            parity.check_measure(M.cpu().numpy(), orc.exact_measure(inp["Q"], inp["K"], inp["lengths"]), inp["lengths"])
+            plan.close()
+        elif mode == 1:    # mean(V)
+            T = int(rng.integers(1, 5000))
+            lengths = [int(rng.integers(0, T + 1)) if rng.random() < 0.7 else T for _ in range(B)]
+            what.update(T=T, lengths=lengths)
+            inp = _synth(B, H, T, 200 + it, 4, dtype, [max(1, L) for L in lengths])
+            inp["lengths"] = np.asarray(lengths, dtype=np.int32)
+            dev, tdt = _dev(inp, dtype)
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c)
+            vb = plan.psattn_mean_v(dev["V"], dev["lengths"])
+            torch.cuda.synchronize()
+            ref = orc.mean_v(inp["V"], inp["lengths"])
+            assert np.abs(vb.cpu().numpy() - ref).max() <= 1e-4, what
+            plan.close()
+        elif mode == 2:    # measure alone, long and ragged
+            T = int(rng.integers(1101, 9000)); B = min(B, 2); H = min(H, 3)
+            lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+            what.update(T=T, lengths=lengths, B=B, H=H)
+            n = max(orc.count(c, L) for L in range(1, T + 1))
+            inp = _synth(B, H, T, 300 + it, n, dtype, lengths)
+            dev, tdt = _dev(inp, dtype)
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n, path=path)
+            M = plan.psattn_measure(dev["Q"], dev["K"], dev["lengths"], dev["sample_idx"]); torch.cuda.synchronize()
+            assert plan.psattn_read_status() == 0
+            parity.check_measure(M.cpu().numpy(), orc.measure(inp["Q"], inp["K"], inp["sample_idx"], inp["lengths"], c=c), inp["lengths"])
+            plan.close()
+        elif mode == 3:    # row lists over long sequences (key splits and their merge)
+            T = int(rng.integers(1500, 9000)); B = min(B, 2); H = min(H, 3)
+            lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.5 else T for _ in range(B)]
+            what.update(T=T, lengths=lengths, B=B, H=H)
+            inp = _synth(B, H, T, 400 + it, 4, dtype, lengths)
+            dev, tdt = _dev(inp, dtype)
+            u_over = int(rng.integers(65, 200)) if (dtype == "bf16" and rng.random() < 0.4) else 0
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c, u_override=u_over, path=path)
+            n_rows = int(rng.integers(1, plan.u_max + 1))
+            rows = np.stack([[rng.integers(0, lengths[b], size=n_rows) for _ in range(H)] for b in range(B)]).astype(np.int32)
+            out = plan.psattn_attend_rows(dev["Q"], dev["K"], dev["V"], dev["lengths"], torch.from_numpy(rows).cuda())
+            torch.cuda.synchronize(); out = out.cpu().numpy()
+            assert plan.psattn_read_status() == 0
+            tol = 1e-4 if dtype == "fp32" else 8e-3
+            for b in range(B):
+                for h in range(H):
+                    for r in rng.choice(n_rows, size=min(n_rows, 3), replace=False):
+                        ref = orc.attend_row(inp["Q"], inp["K"], inp["V"], b, h, int(rows[b, h, r]), lengths[b])
+                        assert np.abs(out[b, h, r] - ref).max() <= tol, ("row", b, h, r)
+            plan.close()
+        else:              # host buffers
+            T = int(rng.choice([rng.integers(1, 300), rng.integers(1101, 2500)])); B = int(rng.integers(1, 6))
+            lengths = [int(rng.integers(1, T + 1)) if rng.random() < 0.6 else T for _ in range(B)]
+            what.update(T=T, lengths=lengths, B=B)
+            n = max(orc.count(c, L) for L in range(1, T + 1))
+            inp = _synth(B, H, T, 500 + it, n, "bf16", lengths)
+            tdt = torch.bfloat16
+            plan = ps.Plan(B, H, T, dtype=tdt, c=c, idx_cols=n, path=path)
+            plan.psattn_plan_enable_host_io()
+            hQ, hK, hV = (torch.from_numpy(inp[k]).to(tdt).pin_memory() for k in ("Q", "K", "V"))
+            hl = torch.from_numpy(inp["lengths"]).pin_memory(); hi = torch.from_numpy(inp["sample_idx"]).pin_memory()
+            hO = torch.empty((B, H, T, 64), dtype=tdt).pin_memory(); hs = torch.empty((B, H, plan.u_max), dtype=torch.int32).pin_memory()
+            plan.psattn_forward_host(hQ, hK, hV, hl, hi, hO, hs)
+            parity.check_forward(hO.float().numpy(), hs.numpy(), None, inp, inp["lengths"], "bf16", c)
+            plan.close()
+

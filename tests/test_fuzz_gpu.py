@@ -344,3 +344,14 @@ def test_random_calls_of_the_other_entry_points_match_the_oracle(seed):
             parity.check_forward(hO.float().numpy(), hs.numpy(), None, inp, inp["lengths"], "bf16", c)
             plan.close()
 
+
+
+def test_more_units_than_a_grid_dimension_holds():
+    """70 000 units of 16 positions: more than the 65 535 blocks a grid's y or z dimension can number."""
+    B, H, T, c = 8750, 8, 16, 5.0
+    n_cols = max(orc.count(c, L) for L in range(1, T + 1))
+    lengths = [T if b % 3 else T // 2 for b in range(B)]
+    inp = _synth(B, H, T, 5, n_cols, "bf16", lengths)
+    O, sel, M, status = _run_forward(inp, "bf16", c, ps.PSATTN_PATH_AUTO)
+    assert status == 0
+    parity.check_forward(O, sel, M, inp, inp["lengths"], "bf16", c, nthreads=16)

@@ -355,3 +355,15 @@ def test_more_units_than_a_grid_dimension_holds():
     O, sel, M, status = _run_forward(inp, "bf16", c, ps.PSATTN_PATH_AUTO)
     assert status == 0
     parity.check_forward(O, sel, M, inp, inp["lengths"], "bf16", c, nthreads=16)
+
+
+@pytest.mark.parametrize("B,H,T,lengths", [(1, 2, 65536, [65536]), (1, 1, 200000, [199999])])
+def test_very_long_sequences(B, H, T, lengths):
+    """Far beyond the longest named workload: the streaming measure kernel, the selection over ranges (65 536) or over
+    a list too long for shared memory (200 000), many key splits in step (d)."""
+    c = 5.0
+    n_cols = orc.count(c, T)
+    inp = _synth(B, H, T, 6, n_cols, "bf16", lengths)
+    O, sel, M, status = _run_forward(inp, "bf16", c, ps.PSATTN_PATH_AUTO)
+    assert status == 0
+    parity.check_forward(O, sel, M, inp, inp["lengths"], "bf16", c, nthreads=16)
